@@ -1,0 +1,198 @@
+/*
+ * lazyev -- LazyEviction decode / track / evict hot path for NVIDIA B200 (sm_100a).
+ *
+ * One handle serves `units = layers * batch * kv_heads` independent cache units;
+ * unit u = (layer * batch + b) * kv_heads + h.  Every unit holds the same number
+ * of cached tokens n (all sequences were prefilled with the same length and are
+ * decoded in lock step), at most `capacity = max(budget, max_prefill) + window`.
+ *
+ * Conventions
+ *   - Every call returns 0 (LAZYEV_OK) or a negative LAZYEV_E* code; nothing
+ *     throws or aborts.  lazyev_last_error() gives the message of the last
+ *     failure on a handle, lazyev_strerror() names a code.
+ *   - "device pointer" arguments are contiguous arrays in the memory of the GPU
+ *     that was current at lazyev_bind(); activations are bfloat16 (raw 16-bit
+ *     patterns), head_dim = 128 elements per row.
+ *   - The caller owns all device memory and the CUDA stream.  The library
+ *     allocates no device memory at all; it owns only the host-side handle.
+ *   - Calls are asynchronous on the bound stream unless stated otherwise.
+ *     A handle must not be used from two threads at once.
+ *
+ * Device memory layout (described so that callers can size and inspect it)
+ *   kv_pool : pages of 64 tokens; one page = 64 K rows (256 B each) followed by
+ *             64 V rows.  Inside a row the eight-element (16-byte) chunk c of
+ *             token slot r is stored at chunk position c ^ (r & 7) (low three
+ *             bits), which makes a linear bulk copy of a page land in shared
+ *             memory free of ldmatrix bank conflicts.  Slot i of unit u lives
+ *             in physical page page_table[u][i / 64], row i % 64.
+ *   state   : page table, and per unit and slot: TS (int32), MRI (int32),
+ *             original position (int32), last probability (float32).
+ *   scratch : eviction source lists, staging for the host-buffer entry point.
+ */
+#ifndef LAZYEV_H
+#define LAZYEV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lazyev lazyev_t;
+
+enum {
+    LAZYEV_OK = 0,
+    LAZYEV_EINVAL = -1,    /* bad argument (null pointer, unsupported shape, out-of-range value) */
+    LAZYEV_ESTATE = -2,    /* call made in the wrong state (e.g. decode before prefill)           */
+    LAZYEV_ECAPACITY = -3, /* the cache of a unit would grow past its capacity                    */
+    LAZYEV_EDEVICE = -4,   /* a kernel reported a failure in the device status word                */
+    LAZYEV_ECUDA = -5      /* a CUDA runtime call failed                                           */
+};
+
+/* Importance score variants: Eq. (2) of the paper and its two ablations
+ * (the rows "w/o H2" and "w/o H1" of the score ablation table). */
+enum { LAZYEV_SCORE_H1_PLUS_H2 = 0, LAZYEV_SCORE_H1_ONLY = 1, LAZYEV_SCORE_H2_ONLY = 2 };
+
+/*
+ * Create a handle.  The seven parameters are the method's: model shape, KV
+ * budget B, observation window W and importance threshold alpha (Section 4 of
+ * the paper; Algorithm 1's inputs W, B, alpha).  Defaults after create: batch 1,
+ * protected recent tokens = window and no protected initial tokens (the paper's
+ * rule), automatic eviction on, score = H1 + H2, max_prefill = budget.
+ * Errors: EINVAL for head_dim != 128, q_heads not a multiple of kv_heads, more
+ * than 8 query heads per KV head, non-positive sizes, budget <= window,
+ * threshold < 0 or NaN.
+ */
+int lazyev_create(lazyev_t** handle, int layers, int q_heads, int kv_heads, int head_dim,
+                  int budget, int window, float threshold);
+
+/* Configuration; all of these must come before lazyev_bind() except set_budget,
+ * set_auto_evict, set_splits and set_stages, which may be called at any time. */
+int lazyev_set_batch(lazyev_t* h, int batch);
+/* Tokens never evicted: the n_recent newest (paper: W) and the n_initial oldest
+ * (paper: 0).  EINVAL unless n_recent >= 1 and budget > n_recent + n_initial. */
+int lazyev_set_protect(lazyev_t* h, int n_recent, int n_initial);
+/* Longest prompt that will be prefilled; raises the capacity when > budget. */
+int lazyev_set_max_prefill(lazyev_t* h, int n_tokens);
+/* Budget B_t used by the next evictions; n_recent + n_initial < budget_now <= create-time budget. */
+int lazyev_set_budget(lazyev_t* h, int budget_now);
+/* on != 0: lazyev_decode_step() runs the eviction itself when one is due (default). */
+int lazyev_set_auto_evict(lazyev_t* h, int on);
+int lazyev_set_score_mode(lazyev_t* h, int mode);
+/* Number of thread blocks (one cluster) that share one unit in the decode
+ * kernel: 0 = choose automatically, else 1, 2, 4 or 8. */
+int lazyev_set_splits(lazyev_t* h, int splits);
+/* Depth of the decode kernel's shared-memory page ring: 0 = as deep as fits, else 2..6. */
+int lazyev_set_stages(lazyev_t* h, int stages);
+
+/* Bytes the caller must provide to lazyev_bind(); any output pointer may be NULL. */
+int lazyev_query_sizes(const lazyev_t* h, size_t* kv_bytes, size_t* state_bytes, size_t* scratch_bytes);
+
+/*
+ * Attach caller-owned device memory (each region at least the size reported by
+ * lazyev_query_sizes and 256-byte aligned) and a CUDA stream (cudaStream_t
+ * passed as void*, NULL = the legacy default stream).  Zeroes the pool, builds
+ * the identity page table and clears the state; asynchronous on the stream.
+ * Errors: EINVAL (null / misaligned), ESTATE (already bound), ECUDA.
+ */
+int lazyev_bind(lazyev_t* h, void* kv_pool, void* state, void* scratch, void* cuda_stream);
+
+/* Replace the page table: host array [units * pages_per_unit] holding a
+ * permutation of 0 .. units*pages_per_unit-1.  Only between bind and prefill. */
+int lazyev_set_page_table(lazyev_t* h, const int32_t* host_table);
+
+/*
+ * Load the prompt's keys and values: device pointers, bf16,
+ * [layers, batch, kv_heads, n_tokens, head_dim].  Sets TS = 0, MRI = 0,
+ * position = 0..n_tokens-1 and the step counter t = 0.
+ * Errors: ESTATE (not bound, or already prefilled), EINVAL, ECAPACITY
+ * (n_tokens > max_prefill).
+ */
+int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens);
+
+/*
+ * One decode step for all units (Algorithm 1 without its last branch unless
+ * automatic eviction is on):
+ *   t += 1; the new token (k_new, v_new) is appended with TS = t, MRI = 0;
+ *   out = softmax(q K^T / sqrt(head_dim)) V over all cached tokens (Eq. attn);
+ *   each cached token's probability, averaged over the query heads of its KV
+ *   group, is stored; tokens whose probability is >= threshold get
+ *   MRI = max(MRI, t - TS), TS = t (Eq. 1).
+ * q, out: [layers, batch, q_heads, head_dim]; k_new, v_new: [layers, batch,
+ * kv_heads, head_dim]; all device pointers, bf16.
+ * Errors: ESTATE (no prefill), ECAPACITY (cache full: eviction was disabled
+ * and never called), ECUDA.  Failures that kernels detect (a bounded wait that
+ * gave up, an index out of range) are recorded in a device status word and
+ * reported by lazyev_synchronize() and lazyev_dump_state() as EDEVICE.
+ */
+int lazyev_decode_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out);
+
+/* The same step with HOST buffers (pinned memory recommended): copies the three
+ * inputs to the device, runs the step, copies `out` back and synchronises the stream. */
+int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out);
+
+/*
+ * Lagged eviction (Section 4 "MRI-Centric Eviction", Eq. 2, Eq. evic): if t is
+ * a multiple of the window and n > budget_now, score every unprotected token,
+ * keep the budget_now - n_recent - n_initial best (ties: the more recent
+ * token) plus the protected ones, and compact K, V, TS, MRI and positions to
+ * the front of each unit in generation order; n becomes budget_now.
+ * Otherwise does nothing and returns 0.  `*evicted` (optional) receives the
+ * number of tokens removed per unit.
+ */
+int lazyev_evict(lazyev_t* h, int* evicted);
+
+typedef struct lazyev_info {
+    int layers, batch, q_heads, kv_heads, head_dim, units;
+    int budget, budget_now, window, n_recent, n_initial;
+    int capacity;        /* slots per unit (multiple of 64)                  */
+    int pages_per_unit;
+    int t;               /* decode steps done                                */
+    int n;               /* cached tokens per unit                           */
+    int prefill;         /* prompt length                                    */
+    int splits;          /* blocks per unit used by the last decode launch   */
+    int stages;          /* pipeline stages used by the last decode launch   */
+    int grid;            /* blocks launched by the last decode launch        */
+    int smem_bytes;      /* dynamic shared memory of the last decode launch  */
+    long long launches;  /* kernels launched by this handle so far           */
+    long long evictions; /* eviction events so far                           */
+} lazyev_info_t;
+
+int lazyev_get_info(const lazyev_t* h, lazyev_info_t* out);
+
+/*
+ * Snapshot for tests and checkpoints; synchronises the stream.  The caller
+ * fills unit_begin / unit_count and the host pointers it wants (NULL = skip);
+ * arrays are [unit_count][capacity] (k, v: [unit_count][capacity][head_dim],
+ * de-swizzled bf16 bits), valid in the first `n` slots of each unit.
+ * `score` receives Eq. (2) evaluated now, at step t, for every cached token.
+ * `device_status` is the kernels' status word (0 = healthy).
+ */
+typedef struct lazyev_dump {
+    int unit_begin, unit_count;                 /* in  */
+    int t, n, capacity, device_status;          /* out */
+    int32_t* pos;
+    int32_t* ts;
+    int32_t* mri;
+    float* pbar;
+    double* score;
+    uint16_t* k;
+    uint16_t* v;
+} lazyev_dump_t;
+
+int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* dump);
+
+/* Waits for the stream and reads the device status word: 0, EDEVICE or ECUDA. */
+int lazyev_synchronize(lazyev_t* h);
+
+/* Frees the host-side handle.  Device memory stays with the caller. */
+int lazyev_destroy(lazyev_t* h);
+
+const char* lazyev_strerror(int code);
+const char* lazyev_last_error(const lazyev_t* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAZYEV_H */

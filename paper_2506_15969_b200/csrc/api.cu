@@ -1,0 +1,510 @@
+// C-ABI layer: host-side handle, argument validation, step / eviction schedule, launches.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <map>
+#include <utility>
+#include <vector>
+
+#include "../../include/lazyev.h"
+#include "internal.h"
+
+using namespace lzk;
+
+struct lazyev {
+    // configuration
+    int layers = 0, batch = 1, q_heads = 0, kv_heads = 0, head_dim = 0;
+    int budget = 0, budget_now = 0, window = 0, n_recent = 0, n_initial = 0, max_prefill = 0;
+    float alpha = 0.f;
+    int auto_evict = 1, score_mode = LAZYEV_SCORE_H1_PLUS_H2, force_splits = 0, force_stages = 0;
+    // derived at bind
+    bool bound = false, prefilled = false;
+    int units = 0, group = 0, capacity = 0, pages_per_unit = 0;
+    int device = -1, num_sms = 0, max_smem = 0;
+    cudaStream_t stream = nullptr;
+    uint8_t* pool = nullptr;
+    StateView st = {};
+    int32_t* src = nullptr;
+    int32_t* first_moved = nullptr;
+    uint8_t* stage_q = nullptr;
+    uint8_t* stage_k = nullptr;
+    uint8_t* stage_v = nullptr;
+    uint8_t* stage_out = nullptr;
+    double* stage_score = nullptr;
+    // progress
+    int t = 0, n = 0, prefill = 0;
+    long long launches = 0, evictions = 0;
+    DecodePlan last_plan = {};
+    int last_grid = 0;
+    std::map<std::pair<int, int>, int> cluster_cache;      // (splits, smem bytes) -> resident clusters
+    char err[256] = {0};
+};
+
+namespace {
+
+constexpr int kScoreStageUnits = 32;      // units whose scores one dump pass evaluates
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int fail(lazyev_t* h, int code, const char* fmt, ...) {
+    if (h) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(h->err, sizeof(h->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+int cuda_fail(lazyev_t* h, cudaError_t e, const char* what) {
+    return fail(h, LAZYEV_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+void derive(lazyev_t* h) {
+    h->units = h->layers * h->batch * h->kv_heads;
+    h->group = h->q_heads / h->kv_heads;
+    const int cap = (h->budget > h->max_prefill ? h->budget : h->max_prefill) + h->window;
+    h->pages_per_unit = (cap + kPageTokens - 1) / kPageTokens;
+    h->capacity = h->pages_per_unit * kPageTokens;
+}
+
+struct Sizes {
+    size_t kv, state, scratch;
+    size_t off_ts, off_mri, off_pos, off_pbar, off_status;                          // inside state
+    size_t off_first, off_q, off_k, off_v, off_out, off_score;                      // inside scratch
+};
+
+Sizes sizes_of(const lazyev_t* h) {
+    Sizes s;
+    const size_t slots = (size_t)h->units * h->capacity;
+    s.kv = (size_t)h->units * h->pages_per_unit * kPageBytes;
+    size_t off = align_up((size_t)h->units * h->pages_per_unit * sizeof(int32_t), 256);
+    s.off_ts = off;
+    off += align_up(slots * 4, 256);
+    s.off_mri = off;
+    off += align_up(slots * 4, 256);
+    s.off_pos = off;
+    off += align_up(slots * 4, 256);
+    s.off_pbar = off;
+    off += align_up(slots * 4, 256);
+    s.off_status = off;
+    off += 256;
+    s.state = off;
+    off = align_up((size_t)h->units * h->budget * sizeof(int32_t), 256);
+    s.off_first = off;
+    off += align_up((size_t)h->units * sizeof(int32_t), 256);
+    const size_t qbytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
+    const size_t kbytes = (size_t)h->layers * h->batch * h->kv_heads * kRowBytes;
+    s.off_q = off;
+    off += align_up(qbytes, 256);
+    s.off_k = off;
+    off += align_up(kbytes, 256);
+    s.off_v = off;
+    off += align_up(kbytes, 256);
+    s.off_out = off;
+    off += align_up(qbytes, 256);
+    s.off_score = off;
+    off += align_up((size_t)kScoreStageUnits * h->capacity * sizeof(double), 256);
+    s.scratch = off;
+    return s;
+}
+
+Geometry geometry(const lazyev_t* h) { return Geometry{h->units, h->group, h->pages_per_unit, h->capacity}; }
+
+int check_device_status(lazyev_t* h) {
+    int32_t status = 0;
+    cudaError_t e = cudaMemcpyAsync(&status, h->st.status, sizeof(status), cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "reading the device status word");
+    if (status != 0) return fail(h, LAZYEV_EDEVICE, "device status word = %d (1: wait timed out, 2: bad index)", status);
+    return LAZYEV_OK;
+}
+
+int run_evict(lazyev_t* h, int* evicted) {
+    if (evicted) *evicted = 0;
+    if (h->t == 0 || h->t % h->window != 0 || h->n <= h->budget_now) return LAZYEV_OK;
+    EvictArgs a;
+    a.n = h->n;
+    a.budget = h->budget_now;
+    a.n_recent = h->n_recent;
+    a.n_initial = h->n_initial;
+    a.t = h->t;
+    a.score_mode = h->score_mode;
+    a.src = h->src;
+    a.first_moved = h->first_moved;
+    if (a.n - a.n_recent - a.n_initial <= 0 || select_smem_bytes(a.n - a.n_recent - a.n_initial) > 200 * 1024)
+        return fail(h, LAZYEV_EINVAL, "eviction over %d candidates is not supported", a.n - a.n_recent - a.n_initial);
+    const Geometry geo = geometry(h);
+    cudaError_t e = select_launch(geo, h->st, a, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "select kernel launch");
+    e = compact_launch(geo, h->pool, h->st, a, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "compact kernel launch");
+    h->launches += 2;
+    h->evictions += 1;
+    if (evicted) *evicted = h->n - h->budget_now;
+    h->n = h->budget_now;
+    return LAZYEV_OK;
+}
+
+int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out) {
+    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
+    if (h->n + 1 > h->capacity) return fail(h, LAZYEV_ECAPACITY, "cache full (%d slots per unit)", h->capacity);
+    const Geometry geo = geometry(h);
+    const int t = h->t + 1, n = h->n + 1;
+    cudaError_t e = append_launch(geo, h->pool, h->st, k_new, v_new, n - 1, t, h->prefill + t - 1, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
+
+    DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages};
+    DecodePlan plan;
+    if (decode_plan(c, n, h->max_smem, h->num_sms, &plan) != 0)
+        return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
+    const std::pair<int, int> key(plan.splits, plan.smem_bytes);
+    auto it = h->cluster_cache.find(key);
+    if (it == h->cluster_cache.end()) {
+        int clusters = 0;
+        e = decode_max_clusters(plan, &clusters);
+        if (e != cudaSuccess) return cuda_fail(h, e, "cluster occupancy query");
+        if (clusters < 1) return fail(h, LAZYEV_ECUDA, "no cluster of %d blocks fits on the device", plan.splits);
+        it = h->cluster_cache.emplace(key, clusters).first;
+    }
+    const int clusters = it->second < h->units ? it->second : h->units;
+    DecodeArgs a{h->pool, h->st, q, out, n, t};
+    e = decode_launch(c, plan, clusters, a, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "decode kernel launch");
+    h->launches += 2;
+    h->last_plan = plan;
+    h->last_grid = clusters * plan.splits;
+    h->t = t;
+    h->n = n;
+    if (h->auto_evict) return run_evict(h, nullptr);
+    return LAZYEV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* lazyev_strerror(int code) {
+    switch (code) {
+        case LAZYEV_OK: return "ok";
+        case LAZYEV_EINVAL: return "invalid argument";
+        case LAZYEV_ESTATE: return "call made in the wrong state";
+        case LAZYEV_ECAPACITY: return "cache capacity exceeded";
+        case LAZYEV_EDEVICE: return "device-side failure flagged";
+        case LAZYEV_ECUDA: return "CUDA runtime error";
+        default: return "unknown error code";
+    }
+}
+
+const char* lazyev_last_error(const lazyev_t* h) { return h ? h->err : "null handle"; }
+
+int lazyev_create(lazyev_t** handle, int layers, int q_heads, int kv_heads, int head_dim, int budget, int window,
+                  float threshold) {
+    if (!handle) return LAZYEV_EINVAL;
+    *handle = nullptr;
+    if (layers <= 0 || q_heads <= 0 || kv_heads <= 0 || budget <= 0 || window <= 0) return LAZYEV_EINVAL;
+    if (head_dim != kHeadDim) return LAZYEV_EINVAL;
+    if (q_heads % kv_heads != 0 || q_heads / kv_heads > kMaxGroup) return LAZYEV_EINVAL;
+    if (budget <= window) return LAZYEV_EINVAL;
+    if (!(threshold >= 0.f)) return LAZYEV_EINVAL;
+    lazyev_t* h = new (std::nothrow) lazyev();
+    if (!h) return LAZYEV_EINVAL;
+    h->layers = layers;
+    h->q_heads = q_heads;
+    h->kv_heads = kv_heads;
+    h->head_dim = head_dim;
+    h->budget = h->budget_now = h->max_prefill = budget;
+    h->window = window;
+    h->n_recent = window;
+    h->alpha = threshold;
+    derive(h);
+    *handle = h;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_batch(lazyev_t* h, int batch) {
+    if (!h) return LAZYEV_EINVAL;
+    if (h->bound) return fail(h, LAZYEV_ESTATE, "set_batch after bind");
+    if (batch <= 0) return fail(h, LAZYEV_EINVAL, "batch must be positive");
+    h->batch = batch;
+    derive(h);
+    return LAZYEV_OK;
+}
+
+int lazyev_set_protect(lazyev_t* h, int n_recent, int n_initial) {
+    if (!h) return LAZYEV_EINVAL;
+    if (h->bound) return fail(h, LAZYEV_ESTATE, "set_protect after bind");
+    if (n_recent < 1 || n_initial < 0 || h->budget <= n_recent + n_initial)
+        return fail(h, LAZYEV_EINVAL, "need n_recent >= 1, n_initial >= 0 and budget > n_recent + n_initial");
+    h->n_recent = n_recent;
+    h->n_initial = n_initial;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_max_prefill(lazyev_t* h, int n_tokens) {
+    if (!h) return LAZYEV_EINVAL;
+    if (h->bound) return fail(h, LAZYEV_ESTATE, "set_max_prefill after bind");
+    if (n_tokens <= 0) return fail(h, LAZYEV_EINVAL, "max_prefill must be positive");
+    h->max_prefill = n_tokens;
+    derive(h);
+    return LAZYEV_OK;
+}
+
+int lazyev_set_budget(lazyev_t* h, int budget_now) {
+    if (!h) return LAZYEV_EINVAL;
+    if (budget_now <= h->n_recent + h->n_initial || budget_now > h->budget)
+        return fail(h, LAZYEV_EINVAL, "budget_now must be in (n_recent + n_initial, budget]");
+    h->budget_now = budget_now;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_auto_evict(lazyev_t* h, int on) {
+    if (!h) return LAZYEV_EINVAL;
+    h->auto_evict = on != 0;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_score_mode(lazyev_t* h, int mode) {
+    if (!h) return LAZYEV_EINVAL;
+    if (mode < 0 || mode > 2) return fail(h, LAZYEV_EINVAL, "unknown score mode %d", mode);
+    h->score_mode = mode;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_splits(lazyev_t* h, int splits) {
+    if (!h) return LAZYEV_EINVAL;
+    if (splits != 0 && splits != 1 && splits != 2 && splits != 4 && splits != 8)
+        return fail(h, LAZYEV_EINVAL, "splits must be 0, 1, 2, 4 or 8");
+    h->force_splits = splits;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_stages(lazyev_t* h, int stages) {
+    if (!h) return LAZYEV_EINVAL;
+    if (stages != 0 && (stages < 2 || stages > 6)) return fail(h, LAZYEV_EINVAL, "stages must be 0 or 2..6");
+    h->force_stages = stages;
+    return LAZYEV_OK;
+}
+
+int lazyev_query_sizes(const lazyev_t* h, size_t* kv_bytes, size_t* state_bytes, size_t* scratch_bytes) {
+    if (!h) return LAZYEV_EINVAL;
+    const Sizes s = sizes_of(h);
+    if (kv_bytes) *kv_bytes = s.kv;
+    if (state_bytes) *state_bytes = s.state;
+    if (scratch_bytes) *scratch_bytes = s.scratch;
+    return LAZYEV_OK;
+}
+
+int lazyev_bind(lazyev_t* h, void* kv_pool, void* state, void* scratch, void* cuda_stream) {
+    if (!h) return LAZYEV_EINVAL;
+    if (h->bound) return fail(h, LAZYEV_ESTATE, "already bound");
+    if (!kv_pool || !state || !scratch) return fail(h, LAZYEV_EINVAL, "null device pointer");
+    if (((uintptr_t)kv_pool | (uintptr_t)state | (uintptr_t)scratch) & 255)
+        return fail(h, LAZYEV_EINVAL, "device regions must be 256-byte aligned");
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e != cudaSuccess) return cuda_fail(h, e, "cudaGetDevice");
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, h->device);
+    if (e != cudaSuccess) return cuda_fail(h, e, "cudaGetDeviceProperties");
+    if (prop.major != 10) return fail(h, LAZYEV_ECUDA, "this library is built for sm_100a only (device is sm_%d%d)", prop.major, prop.minor);
+    h->num_sms = prop.multiProcessorCount;
+    h->max_smem = (int)prop.sharedMemPerBlockOptin;
+    if ((e = decode_prepare()) != cudaSuccess) return cuda_fail(h, e, "decode kernel set-up");
+    if ((e = select_prepare()) != cudaSuccess) return cuda_fail(h, e, "select kernel set-up");
+
+    const Sizes s = sizes_of(h);
+    h->stream = (cudaStream_t)cuda_stream;
+    h->pool = (uint8_t*)kv_pool;
+    uint8_t* sp = (uint8_t*)state;
+    h->st.page_table = (int32_t*)sp;
+    h->st.ts = (int32_t*)(sp + s.off_ts);
+    h->st.mri = (int32_t*)(sp + s.off_mri);
+    h->st.pos = (int32_t*)(sp + s.off_pos);
+    h->st.pbar = (float*)(sp + s.off_pbar);
+    h->st.status = (int32_t*)(sp + s.off_status);
+    uint8_t* cp = (uint8_t*)scratch;
+    h->src = (int32_t*)cp;
+    h->first_moved = (int32_t*)(cp + s.off_first);
+    h->stage_q = cp + s.off_q;
+    h->stage_k = cp + s.off_k;
+    h->stage_v = cp + s.off_v;
+    h->stage_out = cp + s.off_out;
+    h->stage_score = (double*)(cp + s.off_score);
+
+    // Slots past n are read (and masked) by the decode kernel's last page: they must hold finite values.
+    e = cudaMemsetAsync(h->pool, 0, s.kv, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "clearing the KV pool");
+    e = init_state_launch(geometry(h), h->st, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "state initialisation launch");
+    h->launches += 1;
+    h->bound = true;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_page_table(lazyev_t* h, const int32_t* host_table) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!h->bound || h->prefilled) return fail(h, LAZYEV_ESTATE, "set_page_table is only valid between bind and prefill");
+    if (!host_table) return fail(h, LAZYEV_EINVAL, "null page table");
+    const size_t total = (size_t)h->units * h->pages_per_unit;
+    std::vector<char> seen(total, 0);
+    for (size_t i = 0; i < total; ++i) {
+        const int32_t p = host_table[i];
+        if (p < 0 || (size_t)p >= total || seen[p]) return fail(h, LAZYEV_EINVAL, "page table is not a permutation");
+        seen[p] = 1;
+    }
+    cudaError_t e = cudaMemcpyAsync(h->st.page_table, host_table, total * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "page table upload");
+    return LAZYEV_OK;
+}
+
+int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "prefill before bind");
+    if (h->prefilled) return fail(h, LAZYEV_ESTATE, "prefill called twice");
+    if (!k || !v || n_tokens <= 0) return fail(h, LAZYEV_EINVAL, "null pointer or non-positive token count");
+    if (n_tokens > h->max_prefill) return fail(h, LAZYEV_ECAPACITY, "prompt of %d tokens exceeds max_prefill = %d", n_tokens, h->max_prefill);
+    cudaError_t e = prefill_launch(geometry(h), h->pool, h->st, k, v, n_tokens, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill kernel launch");
+    h->launches += 1;
+    h->prefilled = true;
+    h->prefill = n_tokens;
+    h->n = n_tokens;
+    h->t = 0;
+    return LAZYEV_OK;
+}
+
+int lazyev_decode_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!q || !k_new || !v_new || !out) return fail(h, LAZYEV_EINVAL, "null pointer");
+    return run_step(h, q, k_new, v_new, out);
+}
+
+int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!q || !k_new || !v_new || !out) return fail(h, LAZYEV_EINVAL, "null pointer");
+    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
+    const size_t qbytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
+    const size_t kbytes = (size_t)h->layers * h->batch * h->kv_heads * kRowBytes;
+    cudaError_t e = cudaMemcpyAsync(h->stage_q, q, qbytes, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_k, k_new, kbytes, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_v, v_new, kbytes, cudaMemcpyHostToDevice, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "host-to-device copy");
+    const int rc = run_step(h, h->stage_q, h->stage_k, h->stage_v, h->stage_out);
+    if (rc != LAZYEV_OK) return rc;
+    e = cudaMemcpyAsync(out, h->stage_out, qbytes, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "device-to-host copy");
+    return LAZYEV_OK;
+}
+
+int lazyev_evict(lazyev_t* h, int* evicted) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "evict before prefill");
+    return run_evict(h, evicted);
+}
+
+int lazyev_get_info(const lazyev_t* h, lazyev_info_t* out) {
+    if (!h || !out) return LAZYEV_EINVAL;
+    out->layers = h->layers;
+    out->batch = h->batch;
+    out->q_heads = h->q_heads;
+    out->kv_heads = h->kv_heads;
+    out->head_dim = h->head_dim;
+    out->units = h->units;
+    out->budget = h->budget;
+    out->budget_now = h->budget_now;
+    out->window = h->window;
+    out->n_recent = h->n_recent;
+    out->n_initial = h->n_initial;
+    out->capacity = h->capacity;
+    out->pages_per_unit = h->pages_per_unit;
+    out->t = h->t;
+    out->n = h->n;
+    out->prefill = h->prefill;
+    out->splits = h->last_plan.splits;
+    out->stages = h->last_plan.stages;
+    out->grid = h->last_grid;
+    out->smem_bytes = h->last_plan.smem_bytes;
+    out->launches = h->launches;
+    out->evictions = h->evictions;
+    return LAZYEV_OK;
+}
+
+int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* d) {
+    if (!h || !d) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "dump before bind");
+    if (d->unit_begin < 0 || d->unit_count < 0 || d->unit_begin + d->unit_count > h->units)
+        return fail(h, LAZYEV_EINVAL, "unit range out of bounds");
+    d->t = h->t;
+    d->n = h->n;
+    d->capacity = h->capacity;
+    const size_t cap = h->capacity, first = (size_t)d->unit_begin * cap, count = (size_t)d->unit_count * cap;
+    cudaError_t e = cudaSuccess;
+    int32_t status = 0;
+    e = cudaMemcpyAsync(&status, h->st.status, sizeof(status), cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess && d->pos) e = cudaMemcpyAsync(d->pos, h->st.pos + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess && d->ts) e = cudaMemcpyAsync(d->ts, h->st.ts + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess && d->mri) e = cudaMemcpyAsync(d->mri, h->st.mri + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess && d->pbar) e = cudaMemcpyAsync(d->pbar, h->st.pbar + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "state download");
+    if (d->score) {
+        const Geometry geo = geometry(h);
+        for (int u0 = 0; u0 < d->unit_count; u0 += kScoreStageUnits) {
+            const int cnt = d->unit_count - u0 < kScoreStageUnits ? d->unit_count - u0 : kScoreStageUnits;
+            e = score_launch(geo, h->st, d->unit_begin + u0, cnt, h->n, h->t, h->score_mode, h->stage_score, h->stream);
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync(d->score + (size_t)u0 * cap, h->stage_score, (size_t)cnt * cap * sizeof(double), cudaMemcpyDeviceToHost, h->stream);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+            if (e != cudaSuccess) return cuda_fail(h, e, "score download");
+            h->launches += 1;
+        }
+    }
+    if (d->k || d->v) {
+        // Pages come back raw and are un-swizzled here on the host.
+        const int np = (h->n + kPageTokens - 1) / kPageTokens;
+        std::vector<int32_t> table((size_t)d->unit_count * h->pages_per_unit);
+        e = cudaMemcpyAsync(table.data(), h->st.page_table + (size_t)d->unit_begin * h->pages_per_unit, table.size() * 4, cudaMemcpyDeviceToHost, h->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+        if (e != cudaSuccess) return cuda_fail(h, e, "page table download");
+        std::vector<uint8_t> page(kPageBytes);
+        for (int u = 0; u < d->unit_count; ++u) {
+            for (int pg = 0; pg < np; ++pg) {
+                const int32_t pp = table[(size_t)u * h->pages_per_unit + pg];
+                e = cudaMemcpyAsync(page.data(), h->pool + (size_t)pp * kPageBytes, kPageBytes, cudaMemcpyDeviceToHost, h->stream);
+                if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+                if (e != cudaSuccess) return cuda_fail(h, e, "page download");
+                for (int r = 0; r < kPageTokens; ++r) {
+                    const size_t slot = (size_t)u * cap + (size_t)pg * kPageTokens + r;
+                    for (int c = 0; c < kChunksPerRow; ++c) {
+                        const uint8_t* ks = page.data() + r * kRowBytes + swz_chunk(c, r) * 16;
+                        if (d->k) memcpy((uint8_t*)d->k + slot * kRowBytes + c * 16, ks, 16);
+                        if (d->v) memcpy((uint8_t*)d->v + slot * kRowBytes + c * 16, ks + kPageHalfBytes, 16);
+                    }
+                }
+            }
+        }
+    }
+    e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "stream synchronisation");
+    d->device_status = status;
+    if (status != 0) return fail(h, LAZYEV_EDEVICE, "device status word = %d (1: wait timed out, 2: bad index)", status);
+    return LAZYEV_OK;
+}
+
+int lazyev_synchronize(lazyev_t* h) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "synchronize before bind");
+    return check_device_status(h);
+}
+
+int lazyev_destroy(lazyev_t* h) {
+    if (!h) return LAZYEV_EINVAL;
+    delete h;
+    return LAZYEV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,64 @@
+// Host-side interfaces between the C-ABI layer and the kernel launchers.
+#pragma once
+
+#include "common.cuh"
+
+namespace lzk {
+
+// ---- decode ------------------------------------------------------------------
+struct DecodeConfig {
+    int units, group, pages_per_unit, capacity;
+    float alpha;
+    int force_splits;      // 0 = automatic
+    int force_stages;      // 0 = automatic
+};
+
+struct DecodePlan {
+    int splits, stages, pages_per_cta, logit_stride;
+    int off_logits, off_xchg, off_wml, off_misc, off_bars, smem_bytes;
+};
+
+struct DecodeArgs {
+    const uint8_t* pool;
+    StateView state;
+    const void* q;
+    void* out;
+    int n;                 // cached tokens per unit, the new one included
+    int t;                 // this decode step
+};
+
+// Chooses the cluster size, ring depth and shared-memory layout for n cached tokens.
+int decode_plan(const DecodeConfig& c, int n, int max_smem, int num_sms, DecodePlan* plan);
+cudaError_t decode_prepare();
+cudaError_t decode_max_clusters(const DecodePlan& plan, int* clusters);
+cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clusters, const DecodeArgs& a,
+                          cudaStream_t stream);
+
+// ---- cache maintenance ---------------------------------------------------------
+cudaError_t init_state_launch(const Geometry& geo, StateView st, cudaStream_t stream);
+cudaError_t prefill_launch(const Geometry& geo, uint8_t* pool, StateView st, const void* k, const void* v,
+                           int n_tokens, cudaStream_t stream);
+cudaError_t append_launch(const Geometry& geo, uint8_t* pool, StateView st, const void* k_new, const void* v_new,
+                          int slot, int t, int position, cudaStream_t stream);
+
+// ---- eviction --------------------------------------------------------------------
+struct EvictArgs {
+    int n;                 // cached tokens before the eviction
+    int budget;            // tokens to keep (B_t)
+    int n_recent, n_initial;
+    int t;
+    int score_mode;
+    int32_t* src;          // [units][budget]: slot that moves to slot j
+    int32_t* first_moved;  // [units]: first j with src[j] != j (budget if none)
+};
+
+size_t select_smem_bytes(int n_candidates);
+cudaError_t select_prepare();
+cudaError_t select_launch(const Geometry& geo, StateView st, const EvictArgs& a, cudaStream_t stream);
+cudaError_t compact_launch(const Geometry& geo, uint8_t* pool, StateView st, const EvictArgs& a,
+                           cudaStream_t stream);
+// Eq. (2) for every slot < n of units [unit_begin, unit_begin + unit_count) into out[unit][capacity].
+cudaError_t score_launch(const Geometry& geo, StateView st, int unit_begin, int unit_count, int n, int t,
+                         int score_mode, double* out, cudaStream_t stream);
+
+}  // namespace lzk
