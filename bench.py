@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the LazyEviction decode / track / evict hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+A "step" is one pass of the whole hot path over one batch: append the new
+token, decode attention with probability emission and the fused TS / MRI
+update, and -- every W-th step -- the lagged eviction (score, select, compact).
+The default workload is benchmark configuration 4 (batch 32, 28 layers, 28 query
+/ 4 KV heads, head_dim 128, 256-token prompt, budget 8192, window 128) timed in
+its steady state: the real trace is replayed untimed from the prompt up to the
+first eviction (t = 8064), then K steps are timed with the cache cycling between
+8193 and 8320 tokens per unit and one eviction every 128 steps.
+
+Prints one JSON line (rank 0).  `value` is decode tokens/s over all layers with
+inputs resident in HBM; `e2e` is the same through lazyev_decode_step_host with
+pinned host buffers; `roofline` is the decode kernel's algorithmic bytes over
+its CUDA-event time against the measured HBM copy bandwidth; `cpu_baseline` is
+the fp64 oracle on the host cores on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode tokens/sec (all layers, batch B) and fraction of B200 HBM roofline"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch (profiling on small cases)")
+    ap.add_argument("--start-step", type=int, default=-1,
+                    help="decode steps replayed untimed before the timed region (-1: up to the first eviction)")
+    ap.add_argument("--fast-start", action="store_true",
+                    help="prefill a prompt as long as the budget instead of replaying the trace up to it")
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--cpu-units", type=int, default=0)
+    ap.add_argument("--cpu-steps", type=int, default=0)
+    return ap.parse_args()
+
+
+def pick_config(args):
+    from paper_2506_15969_b200 import traces
+    cfg = traces.CONFIGS[args.config]
+    if args.batch:
+        cfg = dataclasses.replace(cfg, batch=args.batch, name=f"{cfg.name}-batch{args.batch}")
+    if args.fast_start:
+        cfg = dataclasses.replace(cfg, prefill=cfg.budget_at(0) if cfg.budget_frac_tenths else cfg.budget,
+                                  name=cfg.name + "-faststart")
+    return cfg
+
+
+def first_eviction_step(cfg) -> int:
+    t = cfg.window
+    while cfg.prefill + t <= cfg.budget_at(t) and t < cfg.steps:
+        t += cfg.window
+    return t
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (no MEASURED_PEAKS.json)"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.stop_flag, self.samples, self.reasons, self.max_mhz = index, False, [], set(), None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+                getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            }
+            while not self.stop_flag:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                time.sleep(0.05)
+        except Exception as e:  # pragma: no cover
+            self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ the oracle leg
+def _oracle_worker(job):
+    """Steps one oracle unit through `steps` decode steps at the benchmark's cache size; returns seconds."""
+    import numpy as np
+    import torch
+    torch.set_num_threads(1)
+    from oracle import lazyev_oracle as orc
+    from paper_2506_15969_b200 import traces
+    cfg, seed, unit, n0, steps, warm = job
+    big = dataclasses.replace(cfg, prefill=n0)
+    gen = traces.TraceGen(big, seed, device="cpu", units=[unit])
+    o = orc.OracleUnit(cfg.group, cfg.head_dim, cfg.budget, cfg.window, cfg.threshold, n_recent=cfg.n_recent,
+                       n_initial=cfg.n_initial)
+    k, v = gen.prefill()
+    o.prefill(k[0].double().numpy(), v[0].double().numpy())
+    spent, done = 0.0, 0
+    while done < warm + steps:
+        cnt = min(32, warm + steps - done)
+        q, kn, vn = gen.steps(cnt)
+        q, kn, vn = q.double().numpy(), kn.double().numpy(), vn.double().numpy()
+        for s in range(cnt):
+            t0 = time.perf_counter()
+            o.step(q[s, 0], kn[s, 0], vn[s, 0])
+            if done >= warm:
+                spent += time.perf_counter() - t0
+            done += 1
+    return spent
+
+
+def time_oracle(cfg, seed, units_sample, n0, steps, warm):
+    """Oracle throughput on the host cores: (tokens/s extrapolated to all units, cores used, description)."""
+    import multiprocessing as mp
+    cores = min(len(units_sample), os.cpu_count() or 1)
+    jobs = [(cfg, seed, u, n0, steps, warm) for u in units_sample]
+    t0 = time.perf_counter()
+    with mp.get_context("spawn").Pool(cores) as pool:
+        spent = pool.map(_oracle_worker, jobs)
+    wall = time.perf_counter() - t0
+    # all sampled units advance `steps` steps in max(spent) seconds on `cores` cores
+    per_step_all_units = max(spent) / steps * (cfg.units / len(units_sample))
+    tokens_per_s = cfg.batch / per_step_all_units
+    sample = (f"{len(units_sample)} of {cfg.units} units x {steps} steps at n~{n0} tokens per unit, one unit per core, "
+              f"extrapolated by units/{len(units_sample)} (setup+run wall {wall:.1f}s)")
+    return tokens_per_s, cores, sample, max(spent) / steps * 1e3
+
+
+def run_reference(args):
+    """The oracle as the reference arm: same metric, bounded sample, host cores only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cfg = pick_config(args)
+    cores = os.cpu_count() or 1
+    units = list(range(0, cfg.units, max(1, cfg.units // cores)))[:cores]
+    n0 = cfg.budget
+    steps = max(1, min(args.steps, 24))
+    tps, used, sample, ms = time_oracle(cfg, args.seed, units, n0, steps, min(args.warmup, 3))
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": cfg.batch / tps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name + " steady state (cache at the budget)", "timed_sample": sample},
+            "cpu_baseline": {"value": tps, "unit": "tokens/s", "cores": used, "kind": "oracle", "sample": sample},
+            "e2e": {"value": tps, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ the CUDA leg
+def run_ours(args):
+    import torch
+    from paper_2506_15969_b200 import binding, traces
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    cfg = pick_config(args)
+    # every rank runs the same per-GPU workload on its own replica of the batch (weak scaling, no exchange)
+    gen = traces.TraceGen(cfg, args.seed + 1000 * rank, device="cuda")
+    eng = binding.Engine(cfg.layers, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window,
+                         cfg.threshold, batch=cfg.batch, n_recent=cfg.n_recent, n_initial=cfg.n_initial,
+                         max_prefill=cfg.prefill)
+    if args.splits:
+        eng.set_splits(args.splits)
+    if args.stages:
+        eng.set_stages(args.stages)
+    L, Bt = cfg.layers, cfg.batch
+    shape = (L, Bt, cfg.kv_heads, cfg.prefill, cfg.head_dim)
+    k, v = gen.prefill()
+    eng.prefill(k.view(shape), v.view(shape))
+    eng.synchronize()
+    del k, v
+    out = torch.empty(L, Bt, cfg.q_heads, cfg.head_dim, dtype=torch.bfloat16, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    t = 0
+
+    def run_chunk(cnt, host=False, timed=False):
+        """Generate `cnt` steps of inputs (untimed), then run them; returns device ms (or wall ms for host)."""
+        nonlocal t
+        q, kn, vn = gen.steps(cnt)
+        if host:
+            qh, kh, vh = q.cpu().pin_memory(), kn.cpu().pin_memory(), vn.cpu().pin_memory()
+            oh = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.perf_counter()
+        e0.record(stream)
+        for s in range(cnt):
+            t += 1
+            if cfg.budget_frac_tenths and t % cfg.window == 0:
+                eng.set_budget(cfg.budget_at(t))
+            if host:
+                eng.decode_step_host(qh[s], kh[s], vh[s], oh)
+            else:
+                eng.decode_step(q[s], kn[s], vn[s], out)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return (time.perf_counter() - w0) * 1e3 if host else e0.elapsed_time(e1)
+
+    def run_steps(count, **kw):
+        ms = 0.0
+        while count > 0:
+            c = min(traces.TraceGen.CHUNK, count)
+            ms += run_chunk(c, **kw)
+            count -= c
+        return ms
+
+    start = first_eviction_step(cfg) if args.start_step < 0 else args.start_step
+    untimed = max(start, args.warmup, 3)
+    run_steps(untimed)                                   # replay + warm-up, not timed
+    eng.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- headline: K steps, inputs resident in HBM, device-timed -------------------
+    sampler = ClockSampler(local)
+    launches0, t_first = eng.info().launches, t + 1
+    barrier()
+    sampler.start()
+    ms = run_steps(args.steps)
+    barrier()
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+    launches = eng.info().launches - launches0
+    evictions_timed = sum(1 for x in range(t_first, t + 1) if x % cfg.window == 0)
+    if dist is not None:
+        tmax = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+    inf = eng.info()
+    value = world * cfg.batch * args.steps / (ms * 1e-3)
+
+    # ---- per-kernel roofline: one observation window with events around each kernel ----
+    roofline, kernels = None, None
+    if not args.no_profile:
+        eng.set_profiling(True)
+        eng.get_profile(reset=True)
+        run_steps(cfg.window)
+        pr = eng.get_profile(reset=True)
+        eng.set_profiling(False)
+        peak, peak_kind = measured_peak()
+        dec_gbs = pr.decode_bytes / (pr.decode_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "decode_kernel (attention + probabilities + TS/MRI update)",
+                    "achieved": round(dec_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
+                    "peak_kind": peak_kind, "frac_of_8TBps_nominal": round(dec_gbs / 8000.0, 4), "traffic": None,
+                    "ms_per_launch": round(pr.decode_ms / max(pr.decode_launches, 1), 4),
+                    "bytes_per_launch": pr.decode_bytes / max(pr.decode_launches, 1)}
+        kernels = {"append_ms_per_launch": round(pr.append_ms / max(pr.append_launches, 1), 4)}
+        if pr.compact_launches:
+            cgbs = pr.compact_bytes / (pr.compact_ms * 1e-3) / 1e9
+            kernels.update({
+                "compact_ms_per_event": round(pr.compact_ms / pr.compact_launches, 4),
+                "compact_GBps": round(cgbs, 1), "compact_frac_of_measured": round(cgbs / peak, 4),
+                "compact_frac_of_8TBps_nominal": round(cgbs / 8000.0, 4),
+                "select_ms_per_event": round(pr.select_ms / pr.select_launches, 4),
+                "select_GBps": round(pr.select_bytes / (pr.select_ms * 1e-3) / 1e9, 1)})
+
+    # ---- end to end: the same steps from pinned host buffers through the C ABI ----------
+    e2e = None
+    if not args.no_e2e:
+        run_steps(3, host=True)
+        e2e_steps = min(args.steps, cfg.window)
+        barrier()
+        wall_ms = run_steps(e2e_steps, host=True)
+        barrier()
+        if dist is not None:
+            tmax = torch.tensor([wall_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            wall_ms = float(tmax.item())
+        qbytes = L * Bt * cfg.q_heads * cfg.head_dim * 2
+        kbytes = L * Bt * cfg.kv_heads * cfg.head_dim * 2
+        e2e = {"value": world * cfg.batch * e2e_steps / (wall_ms * 1e-3), "unit": "tokens/s",
+               "h2d_bytes_per_step": qbytes + 2 * kbytes, "d2h_bytes_per_step": qbytes, "steps": e2e_steps,
+               "ms_per_step": wall_ms / e2e_steps}
+    eng.synchronize()
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, one GPU only) ----------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cores = os.cpu_count() or 1
+        n_units = args.cpu_units or cores
+        sample_units = list(range(0, cfg.units, max(1, cfg.units // n_units)))[:n_units]
+        per_step_est = 6e-6 * inf.n * cfg.group / 7 + 2e-4          # seconds per unit-step, rough
+        steps_cpu = args.cpu_steps or int(max(4, min(16, 2.0 / max(per_step_est, 1e-6))))
+        tps, used, sample, _ = time_oracle(cfg, args.seed, sample_units, inf.budget_now, steps_cpu, 2)
+        cpu = {"value": tps, "unit": "tokens/s", "cores": used, "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: steps {t_first}..{t_first + args.steps - 1} of the seeded trace "
+                                   f"(cache {inf.budget_now}+1..{inf.budget_now}+{cfg.window} tokens per unit, "
+                                   f"{evictions_timed} evictions inside the timed steps)",
+                       "untimed_steps_before": untimed, "units": cfg.units, "batch": cfg.batch, "layers": cfg.layers, "q_heads": cfg.q_heads,
+                       "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget,
+                       "window": cfg.window, "prefill": cfg.prefill, "threshold": cfg.threshold,
+                       "l2": "inputs larger than L2 (KV pool %.1f GB streamed once per step)" % (eng.kv_pool.numel() / 1e9),
+                       "decode_launch": {"splits": inf.splits, "stages": inf.stages, "grid": inf.grid,
+                                         "smem_bytes": inf.smem_bytes},
+                       "multi_gpu": "independent replicas of the batch per GPU, no collective"},
+            "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

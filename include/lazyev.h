@@ -183,6 +183,26 @@ typedef struct lazyev_dump {
 
 int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* dump);
 
+/*
+ * Per-kernel timing for benchmarks.  While profiling is on, every kernel launch
+ * is bracketed by CUDA events on the bound stream (this adds a little latency
+ * between kernels, so headline timings are taken with profiling off).  Times are
+ * summed per kernel; `*_bytes` are the ALGORITHMIC bytes of the same launches:
+ *   decode  : units * (n * (512 + 4) + 2 * group * 256)  -- K/V rows read once,
+ *             one float probability written per token, queries read, outputs written
+ *   select  : units * (8 * candidates + 4 * budget)       -- TS, MRI read; source list written
+ *   compact : moved rows * (2 * (512 + 12) + 4)           -- rows and their state read and written
+ * lazyev_get_profile() synchronises the stream; reset != 0 clears the sums.
+ */
+typedef struct lazyev_profile {
+    double append_ms, decode_ms, select_ms, compact_ms;
+    double decode_bytes, select_bytes, compact_bytes, compact_rows;
+    long long append_launches, decode_launches, select_launches, compact_launches;
+} lazyev_profile_t;
+
+int lazyev_set_profiling(lazyev_t* h, int on);
+int lazyev_get_profile(lazyev_t* h, lazyev_profile_t* out, int reset);
+
 /* Waits for the stream and reads the device status word: 0, EDEVICE or ECUDA. */
 int lazyev_synchronize(lazyev_t* h);
 

@@ -26,6 +26,13 @@ class Info(C.Structure):
         "grid", "smem_bytes")] + [("launches", C.c_longlong), ("evictions", C.c_longlong)]
 
 
+class Profile(C.Structure):
+    _fields_ = [(n, C.c_double) for n in (
+        "append_ms", "decode_ms", "select_ms", "compact_ms", "decode_bytes", "select_bytes", "compact_bytes",
+        "compact_rows")] + [(n, C.c_longlong) for n in (
+            "append_launches", "decode_launches", "select_launches", "compact_launches")]
+
+
 class Dump(C.Structure):
     _fields_ = [("unit_begin", C.c_int), ("unit_count", C.c_int), ("t", C.c_int), ("n", C.c_int),
                 ("capacity", C.c_int), ("device_status", C.c_int),
@@ -52,6 +59,8 @@ _PROTOS = {
     "lazyev_evict": [C.c_void_p, C.POINTER(C.c_int)],
     "lazyev_get_info": [C.c_void_p, C.POINTER(Info)],
     "lazyev_dump_state": [C.c_void_p, C.POINTER(Dump)],
+    "lazyev_set_profiling": [C.c_void_p, C.c_int],
+    "lazyev_get_profile": [C.c_void_p, C.POINTER(Profile), C.c_int],
     "lazyev_synchronize": [C.c_void_p],
     "lazyev_destroy": [C.c_void_p],
 }
@@ -170,6 +179,14 @@ class Engine:
 
     def synchronize(self) -> None:
         self._check(lib().lazyev_synchronize(self._h))
+
+    def set_profiling(self, on: bool) -> None:
+        self._check(lib().lazyev_set_profiling(self._h, int(on)))
+
+    def get_profile(self, reset: bool = False) -> Profile:
+        out = Profile()
+        self._check(lib().lazyev_get_profile(self._h, C.byref(out), int(reset)))
+        return out
 
     def info(self) -> Info:
         out = Info()

@@ -40,6 +40,16 @@ struct lazyev {
     DecodePlan last_plan = {};
     int last_grid = 0;
     std::map<std::pair<int, int>, int> cluster_cache;      // (splits, smem bytes) -> resident clusters
+    // optional per-kernel timing with CUDA events
+    struct Span {
+        cudaEvent_t start, stop;
+        int kind;
+        double bytes;
+    };
+    bool profiling = false;
+    std::vector<Span> pending;
+    std::vector<cudaEvent_t> free_events;
+    lazyev_profile_t prof = {};
     char err[256] = {0};
 };
 
@@ -123,6 +133,59 @@ int check_device_status(lazyev_t* h) {
     return LAZYEV_OK;
 }
 
+enum { kSpanAppend = 0, kSpanDecode = 1, kSpanSelect = 2, kSpanCompact = 3 };
+
+cudaEvent_t take_event(lazyev_t* h) {
+    if (!h->free_events.empty()) {
+        cudaEvent_t e = h->free_events.back();
+        h->free_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+// Brackets one kernel launch with events when profiling is on.
+struct SpanGuard {
+    lazyev_t* h;
+    lazyev::Span span;
+    bool on;
+    SpanGuard(lazyev_t* h_, int kind, double bytes) : h(h_), on(h_->profiling) {
+        if (!on) return;
+        span.start = take_event(h);
+        span.stop = take_event(h);
+        span.kind = kind;
+        span.bytes = bytes;
+        cudaEventRecord(span.start, h->stream);
+    }
+    ~SpanGuard() {
+        if (!on) return;
+        cudaEventRecord(span.stop, h->stream);
+        h->pending.push_back(span);
+    }
+};
+
+int collect_profile(lazyev_t* h) {
+    if (h->pending.empty()) return LAZYEV_OK;
+    cudaError_t e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "stream synchronisation");
+    for (const lazyev::Span& sp : h->pending) {
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, sp.start, sp.stop);
+        switch (sp.kind) {
+            case kSpanAppend: h->prof.append_ms += ms; h->prof.append_launches++; break;
+            case kSpanDecode: h->prof.decode_ms += ms; h->prof.decode_launches++; h->prof.decode_bytes += sp.bytes; break;
+            case kSpanSelect: h->prof.select_ms += ms; h->prof.select_launches++; h->prof.select_bytes += sp.bytes; break;
+            default: h->prof.compact_ms += ms; h->prof.compact_launches++; break;
+        }
+        h->free_events.push_back(sp.start);
+        h->free_events.push_back(sp.stop);
+    }
+    h->pending.clear();
+    return LAZYEV_OK;
+}
+
 int run_evict(lazyev_t* h, int* evicted) {
     if (evicted) *evicted = 0;
     if (h->t == 0 || h->t % h->window != 0 || h->n <= h->budget_now) return LAZYEV_OK;
@@ -138,10 +201,30 @@ int run_evict(lazyev_t* h, int* evicted) {
     if (a.n - a.n_recent - a.n_initial <= 0 || select_smem_bytes(a.n - a.n_recent - a.n_initial) > 200 * 1024)
         return fail(h, LAZYEV_EINVAL, "eviction over %d candidates is not supported", a.n - a.n_recent - a.n_initial);
     const Geometry geo = geometry(h);
-    cudaError_t e = select_launch(geo, h->st, a, h->stream);
+    cudaError_t e;
+    {
+        // algorithmic bytes: TS and MRI of every candidate read, the source list written
+        SpanGuard g(h, kSpanSelect, (double)h->units * (8.0 * (a.n - a.n_recent - a.n_initial) + 4.0 * a.budget));
+        e = select_launch(geo, h->st, a, h->stream);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e, "select kernel launch");
-    e = compact_launch(geo, h->pool, h->st, a, h->stream);
+    {
+        SpanGuard g(h, kSpanCompact, 0.0);
+        e = compact_launch(geo, h->pool, h->st, a, h->stream);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e, "compact kernel launch");
+    if (h->profiling) {
+        // rows that actually moved: every destination from the first evicted slot on
+        std::vector<int32_t> first(h->units);
+        e = cudaMemcpyAsync(first.data(), h->first_moved, first.size() * 4, cudaMemcpyDeviceToHost, h->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+        if (e != cudaSuccess) return cuda_fail(h, e, "first_moved download");
+        double rows = 0;
+        for (int32_t f : first) rows += a.budget - f;
+        // per moved row: K and V rows and three state words read and written, one source index read
+        h->prof.compact_bytes += rows * (2.0 * (2 * kRowBytes + 12) + 4.0);
+        h->prof.compact_rows += rows;
+    }
     h->launches += 2;
     h->evictions += 1;
     if (evicted) *evicted = h->n - h->budget_now;
@@ -154,7 +237,11 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     if (h->n + 1 > h->capacity) return fail(h, LAZYEV_ECAPACITY, "cache full (%d slots per unit)", h->capacity);
     const Geometry geo = geometry(h);
     const int t = h->t + 1, n = h->n + 1;
-    cudaError_t e = append_launch(geo, h->pool, h->st, k_new, v_new, n - 1, t, h->prefill + t - 1, h->stream);
+    cudaError_t e;
+    {
+        SpanGuard g(h, kSpanAppend, 0.0);
+        e = append_launch(geo, h->pool, h->st, k_new, v_new, n - 1, t, h->prefill + t - 1, h->stream);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
 
     DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages};
@@ -172,7 +259,12 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     }
     const int clusters = it->second < h->units ? it->second : h->units;
     DecodeArgs a{h->pool, h->st, q, out, n, t};
-    e = decode_launch(c, plan, clusters, a, h->stream);
+    {
+        // algorithmic bytes: every cached K and V row read once, one probability written per token,
+        // the queries read and the outputs written
+        SpanGuard g(h, kSpanDecode, (double)h->units * ((double)n * (2 * kRowBytes + 4) + 2.0 * h->group * kRowBytes));
+        e = decode_launch(c, plan, clusters, a, h->stream);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e, "decode kernel launch");
     h->launches += 2;
     h->last_plan = plan;
@@ -495,6 +587,23 @@ int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* d) {
     return LAZYEV_OK;
 }
 
+int lazyev_set_profiling(lazyev_t* h, int on) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "set_profiling before bind");
+    const int rc = collect_profile(h);
+    h->profiling = on != 0;
+    return rc;
+}
+
+int lazyev_get_profile(lazyev_t* h, lazyev_profile_t* out, int reset) {
+    if (!h || !out) return LAZYEV_EINVAL;
+    const int rc = collect_profile(h);
+    if (rc != LAZYEV_OK) return rc;
+    *out = h->prof;
+    if (reset) h->prof = lazyev_profile_t{};
+    return LAZYEV_OK;
+}
+
 int lazyev_synchronize(lazyev_t* h) {
     if (!h) return LAZYEV_EINVAL;
     if (!h->bound) return fail(h, LAZYEV_ESTATE, "synchronize before bind");
@@ -503,6 +612,11 @@ int lazyev_synchronize(lazyev_t* h) {
 
 int lazyev_destroy(lazyev_t* h) {
     if (!h) return LAZYEV_EINVAL;
+    for (const lazyev::Span& sp : h->pending) {
+        cudaEventDestroy(sp.start);
+        cudaEventDestroy(sp.stop);
+    }
+    for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
     delete h;
     return LAZYEV_OK;
 }
