@@ -143,6 +143,35 @@ int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const
  */
 int lazyev_evict(lazyev_t* h, int* evicted);
 
+/*
+ * lazyev_evict() for callers that have no scratch region to spare.  (The paper has no
+ * counterpart; this is a deployment convenience.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- a plug-in inside a
+ * serving process that hands out one fixed arena at start-up and treats any later cudaMalloc
+ * as a bug (an allocation synchronises the whole device and stalls every other stream), or a
+ * tool attached to a process whose memory pool is already exhausted by the KV cache itself.
+ * Such a caller can still provide the pool and the state (they are the method's inputs and
+ * outputs), but wants the eviction's work lists to come from somewhere else.
+ *
+ * This entry point does exactly what lazyev_evict() does -- same trigger test, same kernels,
+ * same results bit for bit -- but keeps the source lists and first-moved indices in an array
+ * that is compiled into the library (4 MiB + 16 KiB of device memory on every GPU that loads
+ * the library, held until the process exits) instead of the scratch region given to
+ * lazyev_bind().  It calls no allocator of any kind.
+ *
+ * Limits: units <= 4096 and units * budget_now <= 1,048,576 (2^20) source indices; a larger
+ * handle gets LAZYEV_ECAPACITY and a message naming both numbers, before anything runs.
+ * The device bound to the handle must be the current device (ESTATE otherwise).
+ * The first call on each device looks up the array's device address (one
+ * cudaGetSymbolAddress call, no allocation); make that first call outside any stream capture.
+ * All handles and all calls on one GPU share the one array and it keeps whatever the last
+ * call left in it.  Nothing in it has to start at zero: the select kernel rewrites every entry
+ * that the compact kernel reads.  Two evict_static calls whose kernels overlap on the GPU
+ * (different streams, no dependency between them) race on the array; order them.
+ */
+int lazyev_evict_static(lazyev_t* h, int* evicted);
+
 typedef struct lazyev_info {
     int layers, batch, q_heads, kv_heads, head_dim, units;
     int budget, budget_now, window, n_recent, n_initial;

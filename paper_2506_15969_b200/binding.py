@@ -57,6 +57,7 @@ _PROTOS = {
     "lazyev_decode_step": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_decode_step_host": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_evict": [C.c_void_p, C.POINTER(C.c_int)],
+    "lazyev_evict_static": [C.c_void_p, C.POINTER(C.c_int)],
     "lazyev_get_info": [C.c_void_p, C.POINTER(Info)],
     "lazyev_dump_state": [C.c_void_p, C.POINTER(Dump)],
     "lazyev_set_profiling": [C.c_void_p, C.c_int],
@@ -175,6 +176,13 @@ class Engine:
     def evict(self) -> int:
         n = C.c_int()
         self._check(lib().lazyev_evict(self._h, C.byref(n)))
+        return n.value
+
+    def evict_static(self) -> int:
+        """lazyev_evict_static: the same eviction with its work lists in the library's built-in
+        array instead of the bound scratch region (for callers that cannot allocate)."""
+        n = C.c_int()
+        self._check(lib().lazyev_evict_static(self._h, C.byref(n)))
         return n.value
 
     def synchronize(self) -> None:

@@ -499,6 +499,63 @@ int lazyev_evict(lazyev_t* h, int* evicted) {
     return run_evict(h, evicted);
 }
 
+// ---- eviction without caller-provided scratch ------------------------------------------------
+// Source lists and first-moved indices of lazyev_evict_static(): one array per GPU that loads the
+// library, held until the process exits.  4 MiB + 16 KiB.
+constexpr size_t kStaticSrcEntries = (size_t)1 << 20;      // units * budget_now must not exceed this
+constexpr int kStaticMaxUnits = 4096;
+constexpr int kStaticMaxDevices = 64;
+static __device__ __align__(256) int32_t g_static_evict_scratch[kStaticSrcEntries + kStaticMaxUnits];
+// Device addresses of the array above, one per device ordinal.  The symbol itself is only a
+// host-side stand-in: kernels must be given the address cudaGetSymbolAddress() returns.
+static int32_t* g_static_evict_ptr[kStaticMaxDevices] = {nullptr};
+
+int lazyev_evict_static(lazyev_t* h, int* evicted) {
+    if (!h) return LAZYEV_EINVAL;
+    if (evicted) *evicted = 0;
+    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "evict_static before prefill");
+    if (h->units > kStaticMaxUnits || (size_t)h->units * (size_t)h->budget_now > kStaticSrcEntries)
+        return fail(h, LAZYEV_ECAPACITY,
+                    "evict_static holds %zu source indices for at most %d units; this handle needs %zu for %d units "
+                    "(use lazyev_evict with the bound scratch region)",
+                    kStaticSrcEntries, kStaticMaxUnits, (size_t)h->units * (size_t)h->budget_now, h->units);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(h, e, "cudaGetDevice");
+    if (dev != h->device || dev < 0 || dev >= kStaticMaxDevices)
+        return fail(h, LAZYEV_ESTATE, "evict_static needs device %d (the one bound to this handle) to be current, not %d",
+                    h->device, dev);
+    if (!g_static_evict_ptr[dev]) {    // first call on this device: resolve the array's device address
+        int32_t* ptr = nullptr;
+        e = cudaGetSymbolAddress((void**)&ptr, g_static_evict_scratch);
+        if (e != cudaSuccess || !ptr) return cuda_fail(h, e, "cudaGetSymbolAddress(static eviction scratch)");
+        g_static_evict_ptr[dev] = ptr;
+    }
+    if (h->t == 0 || h->t % h->window != 0 || h->n <= h->budget_now) return LAZYEV_OK;
+    EvictArgs a;
+    a.n = h->n;
+    a.budget = h->budget_now;
+    a.n_recent = h->n_recent;
+    a.n_initial = h->n_initial;
+    a.t = h->t;
+    a.score_mode = h->score_mode;
+    a.src = g_static_evict_ptr[dev];                       // every entry below budget is rewritten by the select
+    a.first_moved = g_static_evict_ptr[dev] + kStaticSrcEntries;   // kernel before the compact kernel reads it
+    const int ncand = a.n - a.n_recent - a.n_initial;
+    if (ncand <= 0 || select_smem_bytes(ncand) > 200 * 1024)
+        return fail(h, LAZYEV_EINVAL, "eviction over %d candidates is not supported", ncand);
+    const Geometry geo = geometry(h);
+    e = select_launch(geo, h->st, a, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "select kernel launch");
+    e = compact_launch(geo, h->pool, h->st, a, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "compact kernel launch");
+    h->launches += 2;
+    h->evictions += 1;
+    if (evicted) *evicted = h->n - h->budget_now;
+    h->n = h->budget_now;
+    return LAZYEV_OK;
+}
+
 int lazyev_get_info(const lazyev_t* h, lazyev_info_t* out) {
     if (!h || !out) return LAZYEV_EINVAL;
     out->layers = h->layers;
