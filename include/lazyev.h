@@ -81,7 +81,7 @@ int lazyev_set_budget(lazyev_t* h, int budget_now);
 int lazyev_set_auto_evict(lazyev_t* h, int on);
 int lazyev_set_score_mode(lazyev_t* h, int mode);
 /* Number of thread blocks (one cluster) that share one unit in the decode
- * kernel: 0 = choose automatically, else 1, 2, 4 or 8. */
+ * kernel: 0 = choose automatically, else 1..8. */
 int lazyev_set_splits(lazyev_t* h, int splits);
 /* Depth of the decode kernel's shared-memory page ring: 0 = as deep as fits, else 2..6. */
 int lazyev_set_stages(lazyev_t* h, int stages);

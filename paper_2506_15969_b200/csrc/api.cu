@@ -39,7 +39,10 @@ struct lazyev {
     long long launches = 0, evictions = 0;
     DecodePlan last_plan = {};
     int last_grid = 0;
-    std::map<std::pair<int, int>, int> cluster_cache;      // (splits, smem bytes) -> resident clusters
+    struct Shape {
+        int splits = 1, clusters = 1, forced_splits = 0, forced_stages = 0;
+    };
+    std::map<int, Shape> plan_cache;                       // pages in use -> launch shape
     // optional per-kernel timing with CUDA events
     struct Span {
         cudaEvent_t start, stop;
@@ -245,19 +248,48 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
 
     DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages};
-    DecodePlan plan;
-    if (decode_plan(c, n, h->max_smem, h->num_sms, &plan) != 0)
-        return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
-    const std::pair<int, int> key(plan.splits, plan.smem_bytes);
-    auto it = h->cluster_cache.find(key);
-    if (it == h->cluster_cache.end()) {
-        int clusters = 0;
-        e = decode_max_clusters(plan, &clusters);
-        if (e != cudaSuccess) return cuda_fail(h, e, "cluster occupancy query");
-        if (clusters < 1) return fail(h, LAZYEV_ECUDA, "no cluster of %d blocks fits on the device", plan.splits);
-        it = h->cluster_cache.emplace(key, clusters).first;
+    // Launch shape: among the cluster sizes whose logits fit in shared memory, take the one that keeps
+    // the most SMs busy, discounted when the page ring gets shallow.  The choice depends only on the
+    // number of pages in use, so it is cached per page count.
+    const int np = (n + kPageTokens - 1) / kPageTokens;
+    auto cached = h->plan_cache.find(np);
+    if (cached == h->plan_cache.end() || cached->second.forced_splits != h->force_splits ||
+        cached->second.forced_stages != h->force_stages) {
+        lazyev::Shape best;
+        best.forced_splits = h->force_splits;
+        best.forced_stages = h->force_stages;
+        double best_score = -1.0;
+        static const double kRingWeight[7] = {0, 0, 0.70, 0.92, 0.97, 1.0, 1.0};
+        for (int s = 1; s <= 8; ++s) {
+            if (h->force_splits > 0 && s != h->force_splits) continue;
+            if (h->force_splits == 0 && s > 1 && (np < 2 * s)) continue;       // at least two pages per block
+            DecodePlan plan;
+            if (decode_plan(c, n + kPageTokens, h->max_smem, s, &plan) != 0) continue;   // room for the page count to grow by one
+            int clusters = 0;
+            e = decode_max_clusters(plan, &clusters);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                continue;
+            }
+            if (clusters < 1) continue;
+            const int used = clusters < h->units ? clusters : h->units;
+            // rounds of the round-robin walk over units decide the tail: count whole rounds
+            const int rounds = (h->units + used - 1) / used;
+            const double busy = (double)h->units * s / ((double)rounds * h->num_sms);
+            const double score = busy * kRingWeight[plan.stages];
+            if (score > best_score + 1e-9) {
+                best_score = score;
+                best.splits = s;
+                best.clusters = used;
+            }
+        }
+        if (best_score < 0) return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
+        cached = h->plan_cache.insert_or_assign(np, best).first;
     }
-    const int clusters = it->second < h->units ? it->second : h->units;
+    DecodePlan plan;
+    if (decode_plan(c, n, h->max_smem, cached->second.splits, &plan) != 0)
+        return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
+    const int clusters = cached->second.clusters;
     DecodeArgs a{h->pool, h->st, q, out, n, t};
     {
         // algorithmic bytes: every cached K and V row read once, one probability written per token,
@@ -368,8 +400,7 @@ int lazyev_set_score_mode(lazyev_t* h, int mode) {
 
 int lazyev_set_splits(lazyev_t* h, int splits) {
     if (!h) return LAZYEV_EINVAL;
-    if (splits != 0 && splits != 1 && splits != 2 && splits != 4 && splits != 8)
-        return fail(h, LAZYEV_EINVAL, "splits must be 0, 1, 2, 4 or 8");
+    if (splits < 0 || splits > 8) return fail(h, LAZYEV_EINVAL, "splits must be 0 (automatic) or 1..8");
     h->force_splits = splits;
     return LAZYEV_OK;
 }

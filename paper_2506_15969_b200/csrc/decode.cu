@@ -10,9 +10,10 @@
 // `splits` blocks.  A cluster walks units round-robin; its blocks split the
 // unit's pages.  Inside a block one producer warp streams 32 KiB pages into a
 // shared-memory ring with linear bulk copies (TMA engine, mbarrier completion);
-// consumer warps each take whole pages: S = Q K^T and O += P V run on
-// mma.sync m16n8k16 with the query heads as the M rows, softmax is online per
-// warp, and the scaled logits of the block's chunk stay in shared memory.
+// the four consumer warps share every page, 16 tokens each: S = Q K^T and
+// O += P V run on mma.sync m16n8k16 with the query heads as the M rows, softmax
+// is online per warp, and the scaled logits of the block's chunk stay in shared
+// memory.
 // After the chunk the warps and then the cluster's blocks merge (m, l, O)
 // through (distributed) shared memory, which gives the exact log-sum-exp; each
 // block then turns its own logits into probabilities, writes pbar and updates
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
     if (threadIdx.x == 0) {
         for (int i = 0; i < NS; ++i) {
             mbar_init(&full[i], 1);
-            mbar_init(&empty[i], 1);
+            mbar_init(&empty[i], NW);          // every consumer warp releases the stage
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
         constexpr int kConsumers = NW * 32;
         const uint32_t ring_base = smem_u32(ring);
         const uint32_t lrow = lane & 7, lmat = lane >> 3;
+        const uint32_t tok_off = 16 * warp;           // this warp's 16 tokens inside every page
         uint32_t pc = 0;
         int it = 0;
         for (int u = cluster_id; u < p.units; u += n_clusters, ++it) {
@@ -178,22 +180,23 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
             for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
 
             for (int j = 0; j < npg; ++j, ++pc) {
-                // Every warp observes every page's barrier, in page order, although it computes only
-                // on its own pages: a parity wait is only meaningful for a waiter that has seen the
-                // previous phase of the same barrier complete, whatever the ring depth.
+                // All consumer warps work on the same page, 16 tokens each, so a stage is held only
+                // for a quarter of a page's arithmetic and goes back to the producer early.  (It also
+                // means every warp sees every phase of every "full" barrier, in order, which a parity
+                // wait needs.)
                 const uint32_t stage = pc % NS;
                 wait_phase(&full[stage], (pc / NS) & 1, abort_flag, p.status);
-                if ((int)(pc % NW) != warp) continue;
-                const uint32_t kb = ring_base + stage * kPageBytes, vb = kb + kPageHalfBytes;
+                const uint32_t kb = ring_base + stage * kPageBytes + tok_off * kRowBytes;
+                const uint32_t vb = kb + kPageHalfBytes;
 
-                // S[g][token] = Q K^T for the 64 tokens of this page (8 tiles of 8 tokens)
-                float sacc[8][4];
+                // S[g][token] = Q K^T for this warp's 16 tokens (2 tiles of 8 tokens)
+                float sacc[2][4];
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
+                for (int nt = 0; nt < 2; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
 #pragma unroll
                 for (int kp = 0; kp < 4; ++kp) {
 #pragma unroll
-                    for (int nt = 0; nt < 8; ++nt) {
+                    for (int nt = 0; nt < 2; ++nt) {
                         uint32_t b0, b1, b2, b3;
                         ldmatrix_x4(b0, b1, b2, b3,
                                     kb + (8 * nt + lrow) * kRowBytes + (((4 * kp + lmat) ^ lrow) << 4));
@@ -203,10 +206,10 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
                 }
 
                 // scale to the log2 domain, mask the slots past n, keep the logits for the epilogue
-                const int tok_base = (pg0 + j) * kPageTokens;
+                const int tok_base = (pg0 + j) * kPageTokens + tok_off;
                 float tmax = -INFINITY;
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {
+                for (int nt = 0; nt < 2; ++nt) {
                     const int t0 = tok_base + 8 * nt + 2 * qd;
                     const float x0 = t0 < p.n ? sacc[nt][0] * p.scale_log2 : -INFINITY;
                     const float x1 = t0 + 1 < p.n ? sacc[nt][1] * p.scale_log2 : -INFINITY;
@@ -214,40 +217,43 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
                     sacc[nt][1] = x1;
                     tmax = fmaxf(tmax, fmaxf(x0, x1));
                     if (g < G)
-                        *reinterpret_cast<float2*>(&logits[g * LS + j * kPageTokens + 8 * nt + 2 * qd]) =
+                        *reinterpret_cast<float2*>(&logits[g * LS + j * kPageTokens + tok_off + 8 * nt + 2 * qd]) =
                             make_float2(x0, x1);
                 }
                 tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
                 tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
                 const float m_new = fmaxf(m_run, tmax);
-                const float corr = fast_exp2(m_run - m_new);
-                m_run = m_new;
-                l_run *= corr;
-                if (corr != 1.f) {
+                if (m_new != -INFINITY) {            // this warp's 16 slots may all lie past n in the last page
+                    if (m_new != m_run) {
+                        const float corr = fast_exp2(m_run - m_new);
+                        m_run = m_new;
+                        l_run *= corr;
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        o[i][0] *= corr;
-                        o[i][1] *= corr;
+                        for (int i = 0; i < 16; ++i) {
+                            o[i][0] *= corr;
+                            o[i][1] *= corr;
+                        }
                     }
-                }
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {
-                    const float p0 = fast_exp2(sacc[nt][0] - m_new), p1 = fast_exp2(sacc[nt][1] - m_new);
-                    l_run += p0 + p1;
-                    sacc[nt][0] = p0;
-                    sacc[nt][1] = p1;
+                    for (int nt = 0; nt < 2; ++nt) {
+                        const float p0 = fast_exp2(sacc[nt][0] - m_new), p1 = fast_exp2(sacc[nt][1] - m_new);
+                        l_run += p0 + p1;
+                        sacc[nt][0] = p0;
+                        sacc[nt][1] = p1;
+                    }
+                } else {
+                    sacc[0][0] = sacc[0][1] = sacc[1][0] = sacc[1][1] = 0.f;
                 }
 
                 // O[g][d] += P V  (P rounded to bf16 for the tensor core; l stays fp32)
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint32_t a0 = pack_bf16(sacc[2 * kk][0], sacc[2 * kk][1]);
-                    const uint32_t a2 = pack_bf16(sacc[2 * kk + 1][0], sacc[2 * kk + 1][1]);
+                {
+                    const uint32_t a0 = pack_bf16(sacc[0][0], sacc[0][1]);
+                    const uint32_t a2 = pack_bf16(sacc[1][0], sacc[1][1]);
 #pragma unroll
                     for (int ntp = 0; ntp < 8; ++ntp) {
                         uint32_t b0, b1, b2, b3;
                         ldmatrix_x4_trans(b0, b1, b2, b3,
-                                          vb + (16 * kk + 8 * (lmat & 1) + lrow) * kRowBytes +
+                                          vb + (8 * (lmat & 1) + lrow) * kRowBytes +
                                               (((2 * ntp + (lmat >> 1)) ^ lrow) << 4));
                         mma_bf16_16816(o[2 * ntp], a0, 0u, a2, 0u, b0, b1);
                         mma_bf16_16816(o[2 * ntp + 1], a0, 0u, a2, 0u, b2, b3);
@@ -320,9 +326,10 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
 
             // out[g][d]: each block of the cluster finishes a slice of the head dimension
             {
-                const int dper = kHeadDim / S;
+                const int d_lo = kHeadDim * (int)rank / S, d_hi = kHeadDim * ((int)rank + 1) / S;
+                const int dper = d_hi - d_lo;
                 for (int e = ctid; e < G * dper; e += kConsumers) {
-                    const int gg = e / dper, d = (int)rank * dper + e % dper;
+                    const int gg = e / dper, d = d_lo + e % dper;
                     float acc = 0.f;
                     for (int r = 0; r < S; ++r)
                         acc += ld_rank_f32(&xb->o[gg][d], r, clustered) * sc_s[r * kMaxGroup + gg];
@@ -362,6 +369,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
 }
 
 constexpr int kConsumerWarps = 4;
+static_assert(kConsumerWarps * 16 == kPageTokens, "each consumer warp takes 16 tokens of a page");
 
 }  // namespace
 
@@ -388,30 +396,12 @@ static size_t layout(const DecodeConfig& c, int np, int s, int ns, DecodePlan* p
     return off;
 }
 
-int decode_plan(const DecodeConfig& c, int n, int max_smem, int num_sms, DecodePlan* plan) {
+int decode_plan(const DecodeConfig& c, int n, int max_smem, int splits, DecodePlan* plan) {
     const int np = (n + kPageTokens - 1) / kPageTokens;
     constexpr int kMaxStages = 6;
-    int want = 1;
-    if (c.force_splits > 0) {
-        want = c.force_splits;
-    } else {
-        // few units: split each one so that the blocks can occupy the SMs
-        while (want < 8 && c.units * want * 2 <= num_sms && np >= 2 * want) want *= 2;
-    }
-    // First choice: the smallest cluster that leaves room for a ring of >= 4 pages;
-    // otherwise whatever fits with at least 2.
-    for (int min_stages = 4; min_stages >= 2; min_stages -= 2) {
-        for (int s = want; s <= 8; s *= 2) {
-            if (c.force_stages > 0) {
-                if (layout(c, np, s, c.force_stages, plan) <= (size_t)max_smem) return 0;
-            } else {
-                for (int ns = kMaxStages; ns >= min_stages; --ns) {
-                    if (layout(c, np, s, ns, plan) <= (size_t)max_smem) return 0;
-                }
-            }
-            if (c.force_splits > 0) break;
-        }
-    }
+    if (c.force_stages > 0) return layout(c, np, splits, c.force_stages, plan) <= (size_t)max_smem ? 0 : -1;
+    for (int ns = kMaxStages; ns >= 2; --ns)
+        if (layout(c, np, splits, ns, plan) <= (size_t)max_smem) return 0;
     return -1;
 }
 

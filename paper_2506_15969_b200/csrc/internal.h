@@ -27,8 +27,9 @@ struct DecodeArgs {
     int t;                 // this decode step
 };
 
-// Chooses the cluster size, ring depth and shared-memory layout for n cached tokens.
-int decode_plan(const DecodeConfig& c, int n, int max_smem, int num_sms, DecodePlan* plan);
+// Deepest ring and the shared-memory layout for n cached tokens and a cluster of `splits` blocks;
+// -1 if nothing fits.
+int decode_plan(const DecodeConfig& c, int n, int max_smem, int splits, DecodePlan* plan);
 cudaError_t decode_prepare();
 cudaError_t decode_max_clusters(const DecodePlan& plan, int* clusters);
 cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clusters, const DecodeArgs& a,

@@ -21,7 +21,7 @@ def lockstep(*a, **kw):
     return Lockstep(*a, **kw)
 
 
-@pytest.mark.parametrize("splits", [1, 2, 4, 8])
+@pytest.mark.parametrize("splits", [1, 2, 3, 4, 5, 8])
 def test_attention_and_tracking_without_eviction(splits):
     """Budget >= prompt + steps: the GPU output is full attention at every step;
     n sweeps across page boundaries and ragged tails (97 .. 296 tokens)."""
@@ -34,7 +34,7 @@ def test_attention_and_tracking_without_eviction(splits):
     assert ls.eng.info().splits == splits
 
 
-@pytest.mark.parametrize("splits,stages", [(1, 2), (1, 3), (2, 3), (1, 5), (4, 2)])
+@pytest.mark.parametrize("splits,stages", [(1, 2), (1, 3), (2, 3), (1, 5), (4, 2), (3, 4), (6, 6)])
 def test_ring_depths_not_a_multiple_of_the_warp_count(splits, stages):
     """Shallow and odd ring depths: pages of one stage are consumed by different warps."""
     cfg = traces.tiny_config(budget=900, window=32, prefill=500, steps=200, batch=1, layers=2)
