@@ -52,6 +52,7 @@ def parse_args():
                     help="prefill a prompt as long as the budget instead of replaying the trace up to it")
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--groups", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
@@ -216,6 +217,8 @@ def run_ours(args):
         eng.set_splits(args.splits)
     if args.stages:
         eng.set_stages(args.stages)
+    if args.groups:
+        eng.set_groups(args.groups)
     L, Bt = cfg.layers, cfg.batch
     shape = (L, Bt, cfg.kv_heads, cfg.prefill, cfg.head_dim)
     k, v = gen.prefill()
@@ -354,7 +357,7 @@ def run_ours(args):
                        "kv_heads": cfg.kv_heads, "head_dim": cfg.head_dim, "budget": cfg.budget,
                        "window": cfg.window, "prefill": cfg.prefill, "threshold": cfg.threshold,
                        "l2": "inputs larger than L2 (KV pool %.1f GB streamed once per step)" % (eng.kv_pool.numel() / 1e9),
-                       "decode_launch": {"splits": inf.splits, "stages": inf.stages, "grid": inf.grid,
+                       "decode_launch": {"splits": inf.splits, "stages": inf.stages, "groups": inf.groups, "grid": inf.grid,
                                          "smem_bytes": inf.smem_bytes},
                        "multi_gpu": "independent replicas of the batch per GPU, no collective"},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),

@@ -68,7 +68,7 @@ int lazyev_create(lazyev_t** handle, int layers, int q_heads, int kv_heads, int 
                   int budget, int window, float threshold);
 
 /* Configuration; all of these must come before lazyev_bind() except set_budget,
- * set_auto_evict, set_splits and set_stages, which may be called at any time. */
+ * set_auto_evict, set_splits, set_stages and set_groups, which may be called at any time. */
 int lazyev_set_batch(lazyev_t* h, int batch);
 /* Tokens never evicted: the n_recent newest (paper: W) and the n_initial oldest
  * (paper: 0).  EINVAL unless n_recent >= 1 and budget > n_recent + n_initial. */
@@ -85,6 +85,9 @@ int lazyev_set_score_mode(lazyev_t* h, int mode);
 int lazyev_set_splits(lazyev_t* h, int splits);
 /* Depth of the decode kernel's shared-memory page ring: 0 = as deep as fits, else 2..6. */
 int lazyev_set_stages(lazyev_t* h, int stages);
+/* Groups of four consumer warps per block in the decode kernel (each group works on
+ * a page of its own): 0 = choose automatically, else 1 or 2. */
+int lazyev_set_groups(lazyev_t* h, int groups);
 
 /* Bytes the caller must provide to lazyev_bind(); any output pointer may be NULL. */
 int lazyev_query_sizes(const lazyev_t* h, size_t* kv_bytes, size_t* state_bytes, size_t* scratch_bytes);
@@ -182,6 +185,7 @@ typedef struct lazyev_info {
     int prefill;         /* prompt length                                    */
     int splits;          /* blocks per unit used by the last decode launch   */
     int stages;          /* pipeline stages used by the last decode launch   */
+    int groups;          /* consumer warp groups used by the last decode launch */
     int grid;            /* blocks launched by the last decode launch        */
     int smem_bytes;      /* dynamic shared memory of the last decode launch  */
     long long launches;  /* kernels launched by this handle so far           */

@@ -23,7 +23,7 @@ class Info(C.Structure):
     _fields_ = [(n, C.c_int) for n in (
         "layers", "batch", "q_heads", "kv_heads", "head_dim", "units", "budget", "budget_now", "window",
         "n_recent", "n_initial", "capacity", "pages_per_unit", "t", "n", "prefill", "splits", "stages",
-        "grid", "smem_bytes")] + [("launches", C.c_longlong), ("evictions", C.c_longlong)]
+        "groups", "grid", "smem_bytes")] + [("launches", C.c_longlong), ("evictions", C.c_longlong)]
 
 
 class Profile(C.Structure):
@@ -50,6 +50,7 @@ _PROTOS = {
     "lazyev_set_score_mode": [C.c_void_p, C.c_int],
     "lazyev_set_splits": [C.c_void_p, C.c_int],
     "lazyev_set_stages": [C.c_void_p, C.c_int],
+    "lazyev_set_groups": [C.c_void_p, C.c_int],
     "lazyev_query_sizes": [C.c_void_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)],
     "lazyev_bind": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_set_page_table": [C.c_void_p, C.c_void_p],
@@ -159,6 +160,9 @@ class Engine:
 
     def set_stages(self, stages: int) -> None:
         self._check(lib().lazyev_set_stages(self._h, stages))
+
+    def set_groups(self, groups: int) -> None:
+        self._check(lib().lazyev_set_groups(self._h, groups))
 
     def set_page_table(self, table) -> None:
         arr = np.ascontiguousarray(np.asarray(table, dtype=np.int32))

@@ -19,7 +19,7 @@ struct lazyev {
     int layers = 0, batch = 1, q_heads = 0, kv_heads = 0, head_dim = 0;
     int budget = 0, budget_now = 0, window = 0, n_recent = 0, n_initial = 0, max_prefill = 0;
     float alpha = 0.f;
-    int auto_evict = 1, score_mode = LAZYEV_SCORE_H1_PLUS_H2, force_splits = 0, force_stages = 0;
+    int auto_evict = 1, score_mode = LAZYEV_SCORE_H1_PLUS_H2, force_splits = 0, force_stages = 0, force_groups = 0;
     // derived at bind
     bool bound = false, prefilled = false;
     int units = 0, group = 0, capacity = 0, pages_per_unit = 0;
@@ -40,7 +40,7 @@ struct lazyev {
     DecodePlan last_plan = {};
     int last_grid = 0;
     struct Shape {
-        int splits = 1, clusters = 1, forced_splits = 0, forced_stages = 0;
+        int splits = 1, clusters = 1, forced_splits = 0, forced_stages = 0, forced_groups = 0;
     };
     std::map<int, Shape> plan_cache;                       // pages in use -> launch shape
     // optional per-kernel timing with CUDA events
@@ -247,17 +247,18 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
 
-    DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages};
+    DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages, h->force_groups};
     // Launch shape: among the cluster sizes whose logits fit in shared memory, take the one that keeps
     // the most SMs busy, discounted when the page ring gets shallow.  The choice depends only on the
     // number of pages in use, so it is cached per page count.
     const int np = (n + kPageTokens - 1) / kPageTokens;
     auto cached = h->plan_cache.find(np);
     if (cached == h->plan_cache.end() || cached->second.forced_splits != h->force_splits ||
-        cached->second.forced_stages != h->force_stages) {
+        cached->second.forced_stages != h->force_stages || cached->second.forced_groups != h->force_groups) {
         lazyev::Shape best;
         best.forced_splits = h->force_splits;
         best.forced_stages = h->force_stages;
+        best.forced_groups = h->force_groups;
         double best_score = -1.0;
         static const double kRingWeight[7] = {0, 0, 0.70, 0.92, 0.97, 1.0, 1.0};
         for (int s = 1; s <= 8; ++s) {
@@ -409,6 +410,13 @@ int lazyev_set_stages(lazyev_t* h, int stages) {
     if (!h) return LAZYEV_EINVAL;
     if (stages != 0 && (stages < 2 || stages > 6)) return fail(h, LAZYEV_EINVAL, "stages must be 0 or 2..6");
     h->force_stages = stages;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_groups(lazyev_t* h, int groups) {
+    if (!h) return LAZYEV_EINVAL;
+    if (groups < 0 || groups > 2) return fail(h, LAZYEV_EINVAL, "groups must be 0 (automatic), 1 or 2");
+    h->force_groups = groups;
     return LAZYEV_OK;
 }
 
@@ -607,6 +615,7 @@ int lazyev_get_info(const lazyev_t* h, lazyev_info_t* out) {
     out->prefill = h->prefill;
     out->splits = h->last_plan.splits;
     out->stages = h->last_plan.stages;
+    out->groups = h->last_plan.groups;
     out->grid = h->last_grid;
     out->smem_bytes = h->last_plan.smem_bytes;
     out->launches = h->launches;

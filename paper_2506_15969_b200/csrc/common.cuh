@@ -141,8 +141,15 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, ui
                  : "r"(addr));
 }
 
-// D += A * B, m16n8k16, bf16 inputs, fp32 accumulate.  Rows 8..15 of A are zero
-// in this library (a1 = a3 = 0), so c[2], c[3] stay zero.
+// Transpose of an 8x8 matrix of 16-bit elements held one 32-bit register per lane
+// (row lane / 4, columns 2 (lane % 4) and the next one).
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
+// D += A * B, m16n8k16, bf16 inputs, fp32 accumulate.
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -162,6 +169,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+
+// The two bf16 halves of a packed pair, widened to fp32 (exact).
+__device__ __forceinline__ float bf16_lo_as_float(uint32_t pair) { return __uint_as_float(pair << 16); }
+__device__ __forceinline__ float bf16_hi_as_float(uint32_t pair) { return __uint_as_float(pair & 0xFFFF0000u); }
 
 __device__ __forceinline__ void named_barrier_sync(int id, int threads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");

@@ -9,14 +9,25 @@
 // Structure: persistent blocks, one block per SM, grouped in clusters of
 // `splits` blocks.  A cluster walks units round-robin; its blocks split the
 // unit's pages.  Inside a block one producer warp streams 32 KiB pages into a
-// shared-memory ring with linear bulk copies (TMA engine, mbarrier completion);
-// the four consumer warps share every page, 16 tokens each: S = Q K^T and
-// O += P V run on mma.sync m16n8k16 with the query heads as the M rows, softmax
-// is online per warp, and the scaled logits of the block's chunk stay in shared
-// memory.
-// After the chunk the warps and then the cluster's blocks merge (m, l, O)
-// through (distributed) shared memory, which gives the exact log-sum-exp; each
-// block then turns its own logits into probabilities, writes pbar and updates
+// shared-memory ring with linear bulk copies (TMA engine, mbarrier completion).
+// Consumer warps come in groups of four; a group takes a whole page, 16 tokens
+// per warp, and with two groups consecutive pages are worked on concurrently.
+//
+// Per 16 tokens a warp runs S^T = K Q^T (tokens are the M rows, query heads the
+// N columns) and O^T += V^T P^T (head dimensions are the M rows) on mma.sync
+// m16n8k16, so both operands that come from the cache fill the whole A tile and
+// the eight query-head columns fill the N = 8 tile.  P goes from the accumulator
+// layout of the first product to the B layout of the second with two movmatrix
+// transposes.  Softmax is online against a per-warp, per-head reference value
+// that is raised (and O, l rescaled) only when a logit exceeds it by more than
+// 2^8, found with one warp vote per tile; any reference gives the same sums.
+//
+// The scaled logits of the block's chunk stay in shared memory (one float per
+// head and token).  After the chunk the warps and then the cluster's blocks
+// merge (reference, l, O) through (distributed) shared memory, which gives the
+// exact log-sum-exp.  The probabilities of a unit are produced while the block's
+// NEXT unit streams: the warp that is about to overwrite the logits of a
+// 16-token tile first turns the old ones into pbar, writes it and updates
 // TS / MRI.  K and V are read from HBM exactly once and nothing but the outputs
 // is written.
 #include "internal.h"
@@ -25,11 +36,11 @@ namespace lzk {
 
 namespace {
 
-constexpr int kXchgRow = kHeadDim + 8;    // padded row of the O exchange buffer (floats)
+constexpr int kXchgRow = kHeadDim + 4;    // row stride = 4 (mod 32) floats: conflict-free fragment stores
 
 struct Xchg {
     float o[kMaxGroup][kXchgRow];         // partial output, relative to m
-    float m[kMaxGroup];                   // running maximum (log2 domain)
+    float m[kMaxGroup];                   // reference value of the partial sums (log2 domain)
     float l[kMaxGroup];                   // sum of exp2(x - m)
 };
 
@@ -50,12 +61,14 @@ struct DecodeParams {
 };
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s is a failure, not a delay
+constexpr float kRaiseMargin = 8.f;                // log2 units a logit may exceed the softmax reference by
 
 // Bounded wait on an mbarrier phase.  On time-out the block-wide abort flag and
 // the device status word are set; once the flag is up no wait blocks any more,
 // so that every thread still reaches the cluster barriers and the kernel ends.
 __device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
                                            bool honour_abort = true) {
+    if (mbar_try_wait(bar, parity)) return true;
     if (honour_abort && *abort_flag) return false;
     uint32_t spins = 0;
     uint64_t t_start = 0;
@@ -80,8 +93,11 @@ __device__ __forceinline__ float ld_rank_f32(const float* local_ptr, uint32_t ra
     return ld_dsmem_f32(map_to_rank(smem_u32(local_ptr), rank));
 }
 
-template <int NW>
-__global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodeParams p) {
+// NG groups of four consumer warps plus one producer warp.
+template <int NG>
+__global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const DecodeParams p) {
+    constexpr int NW = 4 * NG;
+    constexpr int kConsumers = NW * 32;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* ring = smem;
     float* logits = reinterpret_cast<float*>(smem + p.off_logits);
@@ -102,7 +118,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
     if (threadIdx.x == 0) {
         for (int i = 0; i < NS; ++i) {
             mbar_init(&full[i], 1);
-            mbar_init(&empty[i], NW);          // every consumer warp releases the stage
+            mbar_init(&empty[i], 4);           // the four warps of the group that owns the page release it
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -117,6 +133,7 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
     const int pg0 = min(np, (int)rank * p.pages_per_cta);
     const int pg1 = min(np, pg0 + p.pages_per_cta);
     const int npg = pg1 - pg0;
+    const int my_units = cluster_id < p.units ? (p.units - cluster_id + n_clusters - 1) / n_clusters : 0;
 
     if (warp == NW) {
         // ------------------------------------------------------------ producer
@@ -156,150 +173,229 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
         }
     } else {
         // ------------------------------------------------------------ consumers
+        // Fragment coordinates of this lane: row g (and g + 8), column pair 2 qd, 2 qd + 1.
+        // In S^T rows are tokens and columns query heads; in O^T rows are head dimensions.
         const int g = lane >> 2, qd = lane & 3;
+        const int h0 = 2 * qd, h1 = h0 + 1;
+        const bool h0_on = h0 < G, h1_on = h1 < G;
         const int ctid = threadIdx.x;                 // consumer thread id: warps 0..NW-1
-        constexpr int kConsumers = NW * 32;
+        const int grp = warp >> 2, wq = warp & 3;
         const uint32_t ring_base = smem_u32(ring);
-        const uint32_t lrow = lane & 7, lmat = lane >> 3;
-        const uint32_t tok_off = 16 * warp;           // this warp's 16 tokens inside every page
-        uint32_t pc = 0;
+        const uint32_t lrow = lane & 7;
+        // ldmatrix row addresses.  K tile (16 tokens x 16 dims) as the A operand: matrices are
+        // (tokens 0-7, chunk c), (tokens 8-15, c), (tokens 0-7, c + 1), (tokens 8-15, c + 1).
+        // V tile through .trans (16 dims x 16 tokens): (tokens 0-7, c), (tokens 0-7, c + 1),
+        // (tokens 8-15, c), (tokens 8-15, c + 1).
+        const uint32_t tok_off = 16 * wq;             // this warp's 16 tokens inside a page
+        const uint32_t k_lane = (tok_off + (lane & 7) + 8 * ((lane >> 3) & 1)) * kRowBytes, k_sel = lane >> 4;
+        const uint32_t v_lane = kPageHalfBytes + (tok_off + (lane & 7) + 8 * (lane >> 4)) * kRowBytes,
+                       v_sel = (lane >> 3) & 1;
+        const uint32_t pc_total = (uint32_t)my_units * (uint32_t)npg;
+        const int tok0 = pg0 * kPageTokens;           // first token of this block's chunk
+        uint32_t pc = 0;                              // pages of this block, over all its units
+        uint32_t pc_seen = 0;                         // pages whose "full" phase this warp has observed
+        float lse0 = 0.f, lse1 = 0.f;                 // log-sum-exp of the previous unit, heads h0 and h1
+        int u_prev = -1;
         int it = 0;
+
+        // Every warp observes every page's "full" barrier exactly once and in page order: a parity
+        // wait is only valid for a waiter that saw the previous phase of that barrier.
+        auto observe_through = [&](uint32_t last) {
+            for (; pc_seen <= last && pc_seen < pc_total; ++pc_seen)
+                wait_phase(&full[pc_seen % NS], (pc_seen / NS) & 1, abort_flag, p.status);
+        };
+
+        // pbar, TS and MRI of tokens (base + g) and (base + g + 8) of the previous unit from the logits
+        // that are still in shared memory (base: token index inside the block's chunk).
+        auto emit_previous = [&](int base) {
+            float a0 = 0.f, a1 = 0.f;
+            if (h0_on) {
+                a0 = fast_exp2(logits[h0 * LS + base + g] - lse0);
+                a1 = fast_exp2(logits[h0 * LS + base + g + 8] - lse0);
+            }
+            if (h1_on) {
+                a0 += fast_exp2(logits[h1 * LS + base + g] - lse1);
+                a1 += fast_exp2(logits[h1 * LS + base + g + 8] - lse1);
+            }
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 1);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 1);
+            a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
+            a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
+            if (qd == 0) {
+                const size_t row = (size_t)u_prev * p.capacity + tok0;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const int i = base + g + 8 * half;
+                    if (tok0 + i < p.n) {
+                        const float pb = (half ? a1 : a0) * p.inv_group;
+                        p.pbar[row + i] = pb;
+                        if (pb >= p.alpha) {
+                            const int32_t gap = p.t - p.ts[row + i];
+                            if (gap > p.mri[row + i]) p.mri[row + i] = gap;
+                            p.ts[row + i] = p.t;
+                        }
+                    }
+                }
+            }
+        };
+
         for (int u = cluster_id; u < p.units; u += n_clusters, ++it) {
-            uint32_t qa[8][2];
+            // Q^T as the B operand: b0 = Q[head g][16 ks + 2 qd, +1], b1 = the same 8 dims further
+            uint32_t qb[8][2];
             {
                 const __nv_bfloat16* qrow = p.q + ((size_t)u * G + g) * kHeadDim;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    qa[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * qd) : 0u;
-                    qa[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * qd) : 0u;
+                    qb[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * qd) : 0u;
+                    qb[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * qd) : 0u;
                 }
             }
-            float m_run = -INFINITY, l_run = 0.f;
-            float o[16][4];
+            float mref0 = -INFINITY, mref1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+            float o[8][4];      // O^T: [m-tile][(dim g, h0), (dim g, h1), (dim g + 8, h0), (dim g + 8, h1)]
 #pragma unroll
-            for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+            for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
 
             for (int j = 0; j < npg; ++j, ++pc) {
-                // All consumer warps work on the same page, 16 tokens each, so a stage is held only
-                // for a quarter of a page's arithmetic and goes back to the producer early.  (It also
-                // means every warp sees every phase of every "full" barrier, in order, which a parity
-                // wait needs.)
+                if (NG > 1 && (int)(pc % NG) != grp) continue;
+                observe_through(pc);
                 const uint32_t stage = pc % NS;
-                wait_phase(&full[stage], (pc / NS) & 1, abort_flag, p.status);
-                const uint32_t kb = ring_base + stage * kPageBytes + tok_off * kRowBytes;
-                const uint32_t vb = kb + kPageHalfBytes;
+                const uint32_t pb_addr = ring_base + stage * kPageBytes;
+                const int base = j * kPageTokens + (int)tok_off;
 
-                // S[g][token] = Q K^T for this warp's 16 tokens (2 tiles of 8 tokens)
-                float sacc[2][4];
+                // S^T = K Q^T for this warp's 16 tokens, two accumulator chains over the 8 k-steps
+                float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) sacc[nt][0] = sacc[nt][1] = sacc[nt][2] = sacc[nt][3] = 0.f;
-#pragma unroll
-                for (int kp = 0; kp < 4; ++kp) {
-#pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) {
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4(b0, b1, b2, b3,
-                                    kb + (8 * nt + lrow) * kRowBytes + (((4 * kp + lmat) ^ lrow) << 4));
-                        mma_bf16_16816(sacc[nt], qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
-                        mma_bf16_16816(sacc[nt], qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b2, b3);
-                    }
+                for (int ks = 0; ks < 8; ks += 2) {
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4(a0, a1, a2, a3, pb_addr + k_lane + (((2 * ks + k_sel) ^ lrow) << 4));
+                    mma_bf16_16816(sa, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+                    ldmatrix_x4(a0, a1, a2, a3, pb_addr + k_lane + (((2 * ks + 2 + k_sel) ^ lrow) << 4));
+                    mma_bf16_16816(sb, a0, a1, a2, a3, qb[ks + 1][0], qb[ks + 1][1]);
                 }
 
-                // scale to the log2 domain, mask the slots past n, keep the logits for the epilogue
-                const int tok_base = (pg0 + j) * kPageTokens + tok_off;
-                float tmax = -INFINITY;
-#pragma unroll
-                for (int nt = 0; nt < 2; ++nt) {
-                    const int t0 = tok_base + 8 * nt + 2 * qd;
-                    const float x0 = t0 < p.n ? sacc[nt][0] * p.scale_log2 : -INFINITY;
-                    const float x1 = t0 + 1 < p.n ? sacc[nt][1] * p.scale_log2 : -INFINITY;
-                    sacc[nt][0] = x0;
-                    sacc[nt][1] = x1;
-                    tmax = fmaxf(tmax, fmaxf(x0, x1));
-                    if (g < G)
-                        *reinterpret_cast<float2*>(&logits[g * LS + j * kPageTokens + tok_off + 8 * nt + 2 * qd]) =
-                            make_float2(x0, x1);
+                if (it > 0) emit_previous(base);      // the old logits of these slots, before they are overwritten
+
+                // scale to the log2 domain, mask the slots past n, keep the logits for the next pass
+                const bool in0 = tok0 + base + g < p.n, in1 = tok0 + base + g + 8 < p.n;
+                const float x00 = in0 ? (sa[0] + sb[0]) * p.scale_log2 : -INFINITY;     // token g,     head h0
+                const float x01 = in0 ? (sa[1] + sb[1]) * p.scale_log2 : -INFINITY;     // token g,     head h1
+                const float x10 = in1 ? (sa[2] + sb[2]) * p.scale_log2 : -INFINITY;     // token g + 8, head h0
+                const float x11 = in1 ? (sa[3] + sb[3]) * p.scale_log2 : -INFINITY;     // token g + 8, head h1
+                if (h0_on) {
+                    logits[h0 * LS + base + g] = x00;
+                    logits[h0 * LS + base + g + 8] = x10;
                 }
-                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-                const float m_new = fmaxf(m_run, tmax);
-                if (m_new != -INFINITY) {            // this warp's 16 slots may all lie past n in the last page
-                    if (m_new != m_run) {
-                        const float corr = fast_exp2(m_run - m_new);
-                        m_run = m_new;
-                        l_run *= corr;
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            o[i][0] *= corr;
-                            o[i][1] *= corr;
-                        }
-                    }
-#pragma unroll
-                    for (int nt = 0; nt < 2; ++nt) {
-                        const float p0 = fast_exp2(sacc[nt][0] - m_new), p1 = fast_exp2(sacc[nt][1] - m_new);
-                        l_run += p0 + p1;
-                        sacc[nt][0] = p0;
-                        sacc[nt][1] = p1;
-                    }
-                } else {
-                    sacc[0][0] = sacc[0][1] = sacc[1][0] = sacc[1][1] = 0.f;
+                if (h1_on) {
+                    logits[h1 * LS + base + g] = x01;
+                    logits[h1 * LS + base + g + 8] = x11;
                 }
 
-                // O[g][d] += P V  (P rounded to bf16 for the tensor core; l stays fp32)
-                {
-                    const uint32_t a0 = pack_bf16(sacc[0][0], sacc[0][1]);
-                    const uint32_t a2 = pack_bf16(sacc[1][0], sacc[1][1]);
+                // raise the reference only when some logit is more than 2^8 above it (always on the first tile)
+                float mx0 = fmaxf(x00, x10), mx1 = fmaxf(x01, x11);
+                if (__any_sync(0xffffffffu, mx0 > mref0 + kRaiseMargin || mx1 > mref1 + kRaiseMargin)) {
 #pragma unroll
-                    for (int ntp = 0; ntp < 8; ++ntp) {
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4_trans(b0, b1, b2, b3,
-                                          vb + (8 * (lmat & 1) + lrow) * kRowBytes +
-                                              (((2 * ntp + (lmat >> 1)) ^ lrow) << 4));
-                        mma_bf16_16816(o[2 * ntp], a0, 0u, a2, 0u, b0, b1);
-                        mma_bf16_16816(o[2 * ntp + 1], a0, 0u, a2, 0u, b2, b3);
+                    for (int s = 4; s < 32; s <<= 1) {
+                        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, s));
+                        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, s));
+                    }
+                    const float n0 = fmaxf(mref0, mx0), n1 = fmaxf(mref1, mx1);
+                    const float c0 = n0 == mref0 ? 1.f : fast_exp2(mref0 - n0);
+                    const float c1 = n1 == mref1 ? 1.f : fast_exp2(mref1 - n1);
+                    mref0 = n0;
+                    mref1 = n1;
+                    l0 *= c0;
+                    l1 *= c1;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        o[i][0] *= c0;
+                        o[i][1] *= c1;
+                        o[i][2] *= c0;
+                        o[i][3] *= c1;
                     }
                 }
+                // a reference of -inf means that every slot seen so far lies past n: all weights are zero
+                const float r0 = mref0 == -INFINITY ? 0.f : mref0, r1 = mref1 == -INFINITY ? 0.f : mref1;
+                const float p00 = fast_exp2(x00 - r0), p01 = fast_exp2(x01 - r1);
+                const float p10 = fast_exp2(x10 - r0), p11 = fast_exp2(x11 - r1);
+                l0 += p00 + p10;
+                l1 += p01 + p11;
+
+                // O^T += V^T P^T.  P enters the tensor core as two bf16 terms, p = hi + lo, so that the
+                // weights carry 16 mantissa bits: with a single bf16 term a dominant token's weight would
+                // be off by up to 2^-9 whenever the reference is not exactly its logit.  l stays fp32.
+                const uint32_t hi0 = pack_bf16(p00, p01), hi1 = pack_bf16(p10, p11);
+                const uint32_t lo0 = pack_bf16(p00 - bf16_lo_as_float(hi0), p01 - bf16_hi_as_float(hi0));
+                const uint32_t lo1 = pack_bf16(p10 - bf16_lo_as_float(hi1), p11 - bf16_hi_as_float(hi1));
+                const uint32_t bh0 = movmatrix_trans(hi0), bh1 = movmatrix_trans(hi1);   // tokens 0-7 / 8-15:
+                const uint32_t bl0 = movmatrix_trans(lo0), bl1 = movmatrix_trans(lo1);   // (k = 2 qd, +1; head g)
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) {
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4_trans(a0, a1, a2, a3, pb_addr + v_lane + (((2 * mt + v_sel) ^ lrow) << 4));
+                    mma_bf16_16816(o[mt], a0, a1, a2, a3, bh0, bh1);
+                    mma_bf16_16816(o[mt], a0, a1, a2, a3, bl0, bl1);
+                }
+                // Before the page goes back, look at the barriers of the other groups' pages up to this
+                // group's next one: the producer cannot reuse their stages while this one is held.
+                if (NG > 1) observe_through(pc + NG - 1);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[stage]);
             }
 
             // ---- merge the warps of this block ---------------------------------
-            l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-            l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-            if (qd == 0) {
-                wml[warp * 16 + g] = m_run;
-                wml[warp * 16 + 8 + g] = l_run;
+#pragma unroll
+            for (int s = 4; s < 32; s <<= 1) {
+                l0 += __shfl_xor_sync(0xffffffffu, l0, s);
+                l1 += __shfl_xor_sync(0xffffffffu, l1, s);
+            }
+            if (g == 0) {
+                wml[warp * 16 + h0] = mref0;
+                wml[warp * 16 + h1] = mref1;
+                wml[warp * 16 + 8 + h0] = l0;
+                wml[warp * 16 + 8 + h1] = l1;
             }
             named_barrier_sync(1, kConsumers);
-            float m_cta = -INFINITY, l_cta = 0.f;
-#pragma unroll
-            for (int w = 0; w < NW; ++w) m_cta = fmaxf(m_cta, wml[w * 16 + g]);
+            float mc0 = -INFINITY, mc1 = -INFINITY, lc0 = 0.f, lc1 = 0.f;
 #pragma unroll
             for (int w = 0; w < NW; ++w) {
-                const float mw = wml[w * 16 + g];
-                l_cta += mw == -INFINITY ? 0.f : wml[w * 16 + 8 + g] * fast_exp2(mw - m_cta);
+                mc0 = fmaxf(mc0, wml[w * 16 + h0]);
+                mc1 = fmaxf(mc1, wml[w * 16 + h1]);
             }
-            const float f = m_run == -INFINITY ? 0.f : fast_exp2(m_run - m_cta);
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const float m0 = wml[w * 16 + h0], m1 = wml[w * 16 + h1];
+                lc0 += m0 == -INFINITY ? 0.f : wml[w * 16 + 8 + h0] * fast_exp2(m0 - mc0);
+                lc1 += m1 == -INFINITY ? 0.f : wml[w * 16 + 8 + h1] * fast_exp2(m1 - mc1);
+            }
+            const float f0 = mref0 == -INFINITY ? 0.f : fast_exp2(mref0 - mc0);
+            const float f1 = mref1 == -INFINITY ? 0.f : fast_exp2(mref1 - mc1);
             Xchg* xb = xchg + (it & 1);
             for (int w = 0; w < NW; ++w) {     // fixed order: the sum is the same in every run
                 if (warp == w) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float2* dst = reinterpret_cast<float2*>(&xb->o[g][8 * i + 2 * qd]);
-                        float2 v = make_float2(o[i][0] * f, o[i][1] * f);
-                        if (w > 0) {
-                            const float2 old = *dst;
-                            v.x += old.x;
-                            v.y += old.y;
+                    for (int mt = 0; mt < 8; ++mt) {
+                        float* d0 = &xb->o[h0][16 * mt + g];
+                        float* d1 = &xb->o[h1][16 * mt + g];
+                        if (w == 0) {
+                            d0[0] = o[mt][0] * f0;
+                            d1[0] = o[mt][1] * f1;
+                            d0[8] = o[mt][2] * f0;
+                            d1[8] = o[mt][3] * f1;
+                        } else {
+                            d0[0] += o[mt][0] * f0;
+                            d1[0] += o[mt][1] * f1;
+                            d0[8] += o[mt][2] * f0;
+                            d1[8] += o[mt][3] * f1;
                         }
-                        *dst = v;
                     }
                 }
                 named_barrier_sync(1, kConsumers);
             }
-            if (warp == 0 && qd == 0) {
-                xb->m[g] = m_cta;
-                xb->l[g] = l_cta;
+            if (warp == 0 && g == 0) {
+                xb->m[h0] = mc0;
+                xb->m[h1] = mc1;
+                xb->l[h0] = lc0;
+                xb->l[h1] = lc1;
             }
             if (clustered) {
                 cluster_arrive();
@@ -323,6 +419,9 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
                 }
             }
             named_barrier_sync(1, kConsumers);
+            lse0 = lse_s[h0];
+            lse1 = lse_s[h1];
+            u_prev = u;
 
             // out[g][d]: each block of the cluster finishes a slice of the head dimension
             {
@@ -336,27 +435,15 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
                     p.out[((size_t)u * G + gg) * kHeadDim + d] = __float2bfloat16_rn(acc);
                 }
             }
+            // No barrier here: lse_s and sc_s are rewritten only after the barriers of the next unit's
+            // merge, the exchange buffer alternates, and every logit slot is read and rewritten by
+            // the same lane (or, across units, on either side of those barriers).
+        }
 
-            // probabilities of this block's tokens, and the statistics update
-            {
-                const int tok0 = pg0 * kPageTokens;
-                const int cn = min(p.n, pg1 * kPageTokens) - tok0;
-                const size_t row = (size_t)u * p.capacity + tok0;
-                for (int i = ctid; i < cn; i += kConsumers) {
-                    float acc = 0.f;
-                    for (int gg = 0; gg < G; ++gg) acc += fast_exp2(logits[gg * LS + i] - lse_s[gg]);
-                    const float pb = acc * p.inv_group;
-                    p.pbar[row + i] = pb;
-                    if (pb >= p.alpha) {
-                        const int32_t ts_old = p.ts[row + i];
-                        const int32_t gap = p.t - ts_old;
-                        const int32_t mri_old = p.mri[row + i];
-                        if (gap > mri_old) p.mri[row + i] = gap;
-                        p.ts[row + i] = p.t;
-                    }
-                }
-            }
-            named_barrier_sync(1, kConsumers);   // logits, lse and scales are free for the next unit
+        // probabilities and statistics of the block's last unit
+        if (it > 0) {
+            for (int j = 0; j < npg; ++j)
+                if (NG == 1 || j % NG == grp) emit_previous(j * kPageTokens + (int)tok_off);
         }
     }
 
@@ -368,28 +455,48 @@ __global__ void __launch_bounds__((NW + 1) * 32, 1) decode_kernel(const DecodePa
     }
 }
 
-constexpr int kConsumerWarps = 4;
-static_assert(kConsumerWarps * 16 == kPageTokens, "each consumer warp takes 16 tokens of a page");
+constexpr int kMaxGroups = 2;
+
+template <int NG>
+cudaError_t launch_impl(const DecodeParams& p, const DecodePlan& plan, int clusters, cudaStream_t stream,
+                        int* max_clusters) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((max_clusters ? 1 : clusters) * plan.splits, 1, 1);
+    cfg.blockDim = dim3((4 * NG + 1) * 32, 1, 1);
+    cfg.dynamicSmemBytes = plan.smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = plan.splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (max_clusters) return cudaOccupancyMaxActiveClusters(max_clusters, decode_kernel<NG>, &cfg);
+    return cudaLaunchKernelEx(&cfg, decode_kernel<NG>, p);
+}
 
 }  // namespace
 
 // Shared-memory layout for a given cluster size and ring depth; returns the total bytes.
 static size_t layout(const DecodeConfig& c, int np, int s, int ns, DecodePlan* plan) {
     const int ppc = (np + s - 1) / s;
-    const int ls = ppc * kPageTokens + 8;      // +8 floats: rows of different heads start in different banks
+    const int ls = ppc * kPageTokens + 4;      // = 4 (mod 32) floats: the rows of a lane's two heads and of the four
+                                               // lanes of a fragment row fall into different banks
     size_t off = (size_t)ns * kPageBytes;
     plan->off_logits = (int)off;
     off += ((size_t)c.group * ls * sizeof(float) + 127) / 128 * 128;
     plan->off_xchg = (int)off;
     off += 2 * sizeof(Xchg);
     plan->off_wml = (int)off;
-    off += kConsumerWarps * 16 * sizeof(float);
+    off += 4 * kMaxGroups * 16 * sizeof(float);
     plan->off_misc = (int)off;
     off += 128 * sizeof(float);
     plan->off_bars = (int)off;
     off += 2 * (size_t)ns * sizeof(uint64_t);
     plan->splits = s;
     plan->stages = ns;
+    plan->groups = c.force_groups > 0 ? c.force_groups : 2;
     plan->pages_per_cta = ppc;
     plan->logit_stride = ls;
     plan->smem_bytes = (int)off;
@@ -399,30 +506,24 @@ static size_t layout(const DecodeConfig& c, int np, int s, int ns, DecodePlan* p
 int decode_plan(const DecodeConfig& c, int n, int max_smem, int splits, DecodePlan* plan) {
     const int np = (n + kPageTokens - 1) / kPageTokens;
     constexpr int kMaxStages = 6;
-    if (c.force_stages > 0) return layout(c, np, splits, c.force_stages, plan) <= (size_t)max_smem ? 0 : -1;
-    for (int ns = kMaxStages; ns >= 2; --ns)
+    const int min_stages = 2;      // a stage per group being worked on      // a stage per group being worked on
+    if (c.force_stages > 0)
+        return c.force_stages >= min_stages && layout(c, np, splits, c.force_stages, plan) <= (size_t)max_smem ? 0 : -1;
+    for (int ns = kMaxStages; ns >= min_stages; --ns)
         if (layout(c, np, splits, ns, plan) <= (size_t)max_smem) return 0;
     return -1;
 }
 
 cudaError_t decode_prepare() {
-    return cudaFuncSetAttribute(decode_kernel<kConsumerWarps>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(decode_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
 }
 
 cudaError_t decode_max_clusters(const DecodePlan& plan, int* clusters) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(plan.splits, 1, 1);
-    cfg.blockDim = dim3((kConsumerWarps + 1) * 32, 1, 1);
-    cfg.dynamicSmemBytes = plan.smem_bytes;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = plan.splits;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaOccupancyMaxActiveClusters(clusters, decode_kernel<kConsumerWarps>, &cfg);
+    DecodeParams none = {};
+    return plan.groups == 2 ? launch_impl<2>(none, plan, 1, nullptr, clusters)
+                            : launch_impl<1>(none, plan, 1, nullptr, clusters);
 }
 
 cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clusters, const DecodeArgs& a,
@@ -455,20 +556,8 @@ cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clu
     p.off_wml = plan.off_wml;
     p.off_misc = plan.off_misc;
     p.off_bars = plan.off_bars;
-
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(clusters * plan.splits, 1, 1);
-    cfg.blockDim = dim3((kConsumerWarps + 1) * 32, 1, 1);
-    cfg.dynamicSmemBytes = plan.smem_bytes;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = plan.splits;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_kernel<kConsumerWarps>, p);
+    return plan.groups == 2 ? launch_impl<2>(p, plan, clusters, stream, nullptr)
+                            : launch_impl<1>(p, plan, clusters, stream, nullptr);
 }
 
 }  // namespace lzk

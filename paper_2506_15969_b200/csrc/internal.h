@@ -11,10 +11,11 @@ struct DecodeConfig {
     float alpha;
     int force_splits;      // 0 = automatic
     int force_stages;      // 0 = automatic
+    int force_groups;      // 0 = automatic; groups of four consumer warps per block (1 or 2)
 };
 
 struct DecodePlan {
-    int splits, stages, pages_per_cta, logit_stride;
+    int splits, stages, groups, pages_per_cta, logit_stride;
     int off_logits, off_xchg, off_wml, off_misc, off_bars, smem_bytes;
 };
 

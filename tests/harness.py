@@ -55,7 +55,8 @@ def make_oracle(cfg: traces.TraceConfig, score_mode="h1+h2") -> orc.OracleUnit:
 
 class Lockstep:
     def __init__(self, cfg: traces.TraceConfig, seed: int, sample_units, splits: int = 0, stages: int = 0,
-                 score_mode: int = 0, page_table=None, pure: bool = True, check_inputs: bool = True):
+                 score_mode: int = 0, page_table=None, pure: bool = True, check_inputs: bool = True,
+                 groups: int = 0):
         self.cfg, self.sample = cfg, list(sample_units)
         self.eng = make_engine(cfg)
         self.eng.set_auto_evict(False)
@@ -63,6 +64,8 @@ class Lockstep:
             self.eng.set_splits(splits)
         if stages:
             self.eng.set_stages(stages)
+        if groups:
+            self.eng.set_groups(groups)
         if score_mode:
             self.eng.set_score_mode(score_mode)
         if page_table is not None:

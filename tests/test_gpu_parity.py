@@ -34,15 +34,56 @@ def test_attention_and_tracking_without_eviction(splits):
     assert ls.eng.info().splits == splits
 
 
+def test_softmax_reference_is_raised_late():
+    """Logits that grow by far more than the 2^8 margin inside one unit, and a dominant token:
+    the lazily raised softmax reference must give the same sums as an exact running maximum."""
+    eng = binding.Engine(1, 4, 1, 128, 400, 32, 0.05, max_prefill=200)
+    from oracle import lazyev_oracle as orc
+    gen = torch.Generator().manual_seed(5)
+    k = torch.randn(200, 128, generator=gen)
+    k *= torch.linspace(0.05, 6.0, 200)[:, None]            # later keys are much longer
+    v = torch.randn(200, 128, generator=gen)
+    q = (torch.randn(4, 128, generator=gen) + 0.8 * k[150] / k[150].norm() * 11.3).to(torch.bfloat16)
+    kb, vb = k.to(torch.bfloat16), v.to(torch.bfloat16)
+    eng.prefill(kb.view(1, 1, 1, 200, 128).cuda(), vb.view(1, 1, 1, 200, 128).cuda())
+    out = torch.empty(1, 1, 4, 128, dtype=torch.bfloat16, device="cuda")
+    kn, vn = torch.randn(1, 128, generator=gen).to(torch.bfloat16), torch.randn(1, 128, generator=gen).to(torch.bfloat16)
+    eng.decode_step(q.view(1, 1, 4, 128).cuda(), kn.view(1, 1, 1, 128).cuda(), vn.view(1, 1, 1, 128).cuda(), out)
+    o = orc.OracleUnit(4, 128, 400, 32, 0.05)
+    o.prefill(kb.double().numpy(), vb.double().numpy())
+    ref_out, ref_pbar = o.attend(q.double().numpy(), kn[0].double().numpy(), vn[0].double().numpy())
+    d = eng.dump_state()
+    assert np.abs(d["pbar"][0] - ref_pbar).max() <= 1e-4
+    assert ref_pbar.max() > 0.05                            # some token really dominates
+    got = out.view(4, 128).double().cpu().numpy()
+    assert (np.abs(got - ref_out) <= 2e-3 + 1e-2 * np.abs(ref_out)).all()
+
+
+@pytest.mark.parametrize("groups", [1, 2])
 @pytest.mark.parametrize("splits,stages", [(1, 2), (1, 3), (2, 3), (1, 5), (4, 2), (3, 4), (6, 6)])
-def test_ring_depths_not_a_multiple_of_the_warp_count(splits, stages):
-    """Shallow and odd ring depths: pages of one stage are consumed by different warps."""
+def test_ring_depths_and_warp_groups(splits, stages, groups):
+    """Shallow and odd ring depths with one and two groups of consumer warps: with two groups a
+    stage's consecutive uses go to different groups, and a block's page count may be odd, so
+    the group that owns a logit tile changes from unit to unit."""
     cfg = traces.tiny_config(budget=900, window=32, prefill=500, steps=200, batch=1, layers=2)
-    ls = lockstep(cfg, seed=11, sample_units=range(cfg.units), splits=splits, stages=stages, pure=False)
+    ls = lockstep(cfg, seed=11, sample_units=range(cfg.units), splits=splits, stages=stages, groups=groups,
+                  pure=False)
     ls.run(150)
     ls.assert_ok()
     inf = ls.eng.info()
-    assert (inf.splits, inf.stages) == (splits, stages)
+    assert (inf.splits, inf.stages, inf.groups) == (splits, stages, groups)
+
+
+@pytest.mark.parametrize("groups", [1, 2])
+def test_many_units_per_block(groups):
+    """More units than blocks: every block walks several units, so the probabilities of one unit are
+    produced while the next one streams, and the last one is flushed at the end."""
+    cfg = traces.tiny_config(batch=40, layers=8, q_heads=14, kv_heads=2, budget=300, window=32, prefill=280)
+    assert cfg.units == 640
+    ls = lockstep(cfg, seed=13, sample_units=[0, 1, 147, 148, 149, 295, 296, 500, 638, 639], groups=groups, pure=False)
+    ls.run(70)
+    ls.assert_ok()
+    assert ls.rep.evictions == 2
 
 
 @pytest.mark.parametrize("q_heads,kv_heads", [(7, 1), (10, 2), (8, 1), (2, 2), (6, 2)])
