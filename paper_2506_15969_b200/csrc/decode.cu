@@ -56,7 +56,7 @@ struct DecodeParams {
     int units, group, pages_per_unit, capacity, total_pages;
     int n, t;
     float alpha, scale_log2, inv_group;
-    int splits, stages, pages_per_cta, logit_stride;
+    int splits, stages, pages_per_cta, logit_stride, tmem_pages, tmem_cols;
     int off_logits, off_xchg, off_wml, off_misc, off_bars;
 };
 
@@ -100,12 +100,13 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
     constexpr int kConsumers = NW * 32;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint8_t* ring = smem;
-    float* logits = reinterpret_cast<float*>(smem + p.off_logits);
+    float* spill = reinterpret_cast<float*>(smem + p.off_logits);       // logits of the pages beyond tensor memory
     Xchg* xchg = reinterpret_cast<Xchg*>(smem + p.off_xchg);          // [2], alternating per unit
     float* wml = reinterpret_cast<float*>(smem + p.off_wml);            // [NW][16]: m[8], l[8] per warp
     float* lse_s = reinterpret_cast<float*>(smem + p.off_misc);         // [8]
     float* sc_s = lse_s + kMaxGroup;                                    // [splits <= 8][8]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sc_s + 8 * kMaxGroup);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sc_s + 8 * kMaxGroup) + 1;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + p.off_bars);
     uint64_t* empty = full + p.stages;
 
@@ -123,7 +124,14 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         *abort_flag = 0;
         fence_barrier_init();
     }
+    if (warp == 0) {                           // tensor memory for the logits: allocated and freed by warp 0
+        tmem_alloc(tmem_slot, (uint32_t)p.tmem_cols);
+        tmem_relinquish_alloc_permit();
+    }
+    tmem_fence_before_sync();
     __syncthreads();
+    tmem_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
     if (clustered) {   // every block of the cluster is resident before any remote access
         cluster_arrive();
         cluster_wait();
@@ -137,7 +145,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 
     if (warp == NW) {
         // ------------------------------------------------------------ producer
-        uint32_t pc = 0;
+        uint32_t pc = 0, stage = 0, parity = 1;     // parity of the "empty" phase that frees the stage
         int it = 0;
         for (int u = cluster_id; u < p.units; u += n_clusters, ++it) {
             const int32_t* pt = p.page_table + (size_t)u * p.pages_per_unit + pg0;
@@ -146,8 +154,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 const int32_t entry = lane < cnt ? pt[base + lane] : 0;
                 for (int j = 0; j < cnt; ++j, ++pc) {
                     int32_t pp = __shfl_sync(0xffffffffu, entry, j);
-                    const uint32_t stage = pc % NS, use = pc / NS;
-                    if (use > 0) wait_phase(&empty[stage], (use - 1) & 1, abort_flag, p.status);
+                    if (pc >= (uint32_t)NS) wait_phase(&empty[stage], parity, abort_flag, p.status);
                     if (lane == 0) {
                         if (pp < 0 || pp >= p.total_pages) {
                             atomicOr(p.status, kStatusBadIndex);
@@ -158,6 +165,10 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                                   &full[stage]);
                     }
                     __syncwarp();
+                    if (++stage == (uint32_t)NS) {
+                        stage = 0;
+                        parity ^= 1;
+                    }
                 }
             }
             if (clustered) {   // this warp's share of the per-unit cluster barrier, split so it can run ahead
@@ -185,15 +196,28 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         // ldmatrix row addresses.  K tile (16 tokens x 16 dims) as the A operand: matrices are
         // (tokens 0-7, chunk c), (tokens 8-15, c), (tokens 0-7, c + 1), (tokens 8-15, c + 1).
         // V tile through .trans (16 dims x 16 tokens): (tokens 0-7, c), (tokens 0-7, c + 1),
-        // (tokens 8-15, c), (tokens 8-15, c + 1).
+        // (tokens 8-15, c), (tokens 8-15, c + 1).  Chunk c of row r sits at c ^ (r & 7): for
+        // k-step ks the lane's byte offset is lane_term ^ (ks << 5); ks bit 2 only adds 128.
         const uint32_t tok_off = 16 * wq;             // this warp's 16 tokens inside a page
-        const uint32_t k_lane = (tok_off + (lane & 7) + 8 * ((lane >> 3) & 1)) * kRowBytes, k_sel = lane >> 4;
-        const uint32_t v_lane = kPageHalfBytes + (tok_off + (lane & 7) + 8 * (lane >> 4)) * kRowBytes,
-                       v_sel = (lane >> 3) & 1;
+        const uint32_t k_row = (tok_off + (lane & 7) + 8 * ((lane >> 3) & 1)) * kRowBytes;
+        const uint32_t v_row = kPageHalfBytes + (tok_off + (lane & 7) + 8 * (lane >> 4)) * kRowBytes;
+        const uint32_t k_term = ((lane >> 4) ^ lrow) << 4, v_term = (((lane >> 3) & 1) ^ lrow) << 4;
+        uint32_t k_off[4], v_off[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            k_off[i] = k_row + (k_term ^ (i << 5));
+            v_off[i] = v_row + (v_term ^ (i << 5));
+        }
+        // Logits of page j of the chunk: tensor-memory columns 4 j .. 4 j + 3 of this thread's lane
+        // (x00, x01, x10, x11), or the shared-memory spill area for the pages beyond tensor memory.
+        const uint32_t tmem_lane = tmem_base + ((uint32_t)(32 * wq) << 16);
+        const int tmem_pages = p.tmem_pages;
         const uint32_t pc_total = (uint32_t)my_units * (uint32_t)npg;
         const int tok0 = pg0 * kPageTokens;           // first token of this block's chunk
-        uint32_t pc = 0;                              // pages of this block, over all its units
-        uint32_t pc_seen = 0;                         // pages whose "full" phase this warp has observed
+        uint32_t pc_base = 0;                         // pages of this block before the current unit
+        uint32_t pc_mod = 0;                          // pc_base mod NG
+        uint32_t st_base = 0, par_base = 0;           // ring stage and "full" parity of page pc_base
+        uint32_t pc_seen = 0, st_seen = 0, par_seen = 0;   // next page whose "full" phase this warp observes
         float lse0 = 0.f, lse1 = 0.f;                 // log-sum-exp of the previous unit, heads h0 and h1
         int u_prev = -1;
         int it = 0;
@@ -201,21 +225,52 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         // Every warp observes every page's "full" barrier exactly once and in page order: a parity
         // wait is only valid for a waiter that saw the previous phase of that barrier.
         auto observe_through = [&](uint32_t last) {
-            for (; pc_seen <= last && pc_seen < pc_total; ++pc_seen)
-                wait_phase(&full[pc_seen % NS], (pc_seen / NS) & 1, abort_flag, p.status);
+            while (pc_seen <= last && pc_seen < pc_total) {
+                wait_phase(&full[st_seen], par_seen, abort_flag, p.status);
+                ++pc_seen;
+                if (++st_seen == (uint32_t)NS) {
+                    st_seen = 0;
+                    par_seen ^= 1;
+                }
+            }
         };
 
-        // pbar, TS and MRI of tokens (base + g) and (base + g + 8) of the previous unit from the logits
-        // that are still in shared memory (base: token index inside the block's chunk).
-        auto emit_previous = [&](int base) {
-            float a0 = 0.f, a1 = 0.f;
-            if (h0_on) {
-                a0 = fast_exp2(logits[h0 * LS + base + g] - lse0);
-                a1 = fast_exp2(logits[h0 * LS + base + g + 8] - lse0);
+        auto load_logits = [&](int j, float& x00, float& x01, float& x10, float& x11) {
+            if (j < tmem_pages) {
+                tmem_ld4(tmem_lane + 4 * j, x00, x01, x10, x11);
+                tmem_wait_ld();
+            } else {
+                const int i = (j - tmem_pages) * kPageTokens + (int)tok_off + g;
+                x00 = h0_on ? spill[h0 * LS + i] : 0.f;
+                x10 = h0_on ? spill[h0 * LS + i + 8] : 0.f;
+                x01 = h1_on ? spill[h1 * LS + i] : 0.f;
+                x11 = h1_on ? spill[h1 * LS + i + 8] : 0.f;
             }
+        };
+        auto store_logits = [&](int j, float x00, float x01, float x10, float x11) {
+            if (j < tmem_pages) {
+                tmem_st4(tmem_lane + 4 * j, x00, x01, x10, x11);
+            } else {
+                const int i = (j - tmem_pages) * kPageTokens + (int)tok_off + g;
+                if (h0_on) {
+                    spill[h0 * LS + i] = x00;
+                    spill[h0 * LS + i + 8] = x10;
+                }
+                if (h1_on) {
+                    spill[h1 * LS + i] = x01;
+                    spill[h1 * LS + i + 8] = x11;
+                }
+            }
+        };
+
+        // pbar, TS and MRI of tokens (base + g) and (base + g + 8) of the previous unit from its logits
+        // (base: token index inside the block's chunk).
+        auto emit_previous = [&](int base, float x00, float x01, float x10, float x11) {
+            float a0 = h0_on ? fast_exp2(x00 - lse0) : 0.f;
+            float a1 = h0_on ? fast_exp2(x10 - lse0) : 0.f;
             if (h1_on) {
-                a0 += fast_exp2(logits[h1 * LS + base + g] - lse1);
-                a1 += fast_exp2(logits[h1 * LS + base + g + 8] - lse1);
+                a0 += fast_exp2(x01 - lse1);
+                a1 += fast_exp2(x11 - lse1);
             }
             a0 += __shfl_xor_sync(0xffffffffu, a0, 1);
             a1 += __shfl_xor_sync(0xffffffffu, a1, 1);
@@ -255,11 +310,17 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 #pragma unroll
             for (int i = 0; i < 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
 
-            for (int j = 0; j < npg; ++j, ++pc) {
-                if (NG > 1 && (int)(pc % NG) != grp) continue;
+            // this group's pages of the unit: j = j0, j0 + NG, ...
+            const int j0 = NG == 1 ? 0 : (int)((grp + NG - pc_mod) % NG);
+            uint32_t stage = st_base + j0, parity = par_base;
+            if (stage >= (uint32_t)NS) {
+                stage -= NS;
+                parity ^= 1;
+            }
+            for (int j = j0; j < npg; j += NG) {
+                const uint32_t pc = pc_base + j;
                 observe_through(pc);
-                const uint32_t stage = pc % NS;
-                const uint32_t pb_addr = ring_base + stage * kPageBytes;
+                const uint32_t page = ring_base + stage * kPageBytes;
                 const int base = j * kPageTokens + (int)tok_off;
 
                 // S^T = K Q^T for this warp's 16 tokens, two accumulator chains over the 8 k-steps
@@ -267,28 +328,28 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 #pragma unroll
                 for (int ks = 0; ks < 8; ks += 2) {
                     uint32_t a0, a1, a2, a3;
-                    ldmatrix_x4(a0, a1, a2, a3, pb_addr + k_lane + (((2 * ks + k_sel) ^ lrow) << 4));
+                    ldmatrix_x4(a0, a1, a2, a3, page + k_off[ks & 3] + 128 * (ks >> 2));
                     mma_bf16_16816(sa, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
-                    ldmatrix_x4(a0, a1, a2, a3, pb_addr + k_lane + (((2 * ks + 2 + k_sel) ^ lrow) << 4));
+                    ldmatrix_x4(a0, a1, a2, a3, page + k_off[(ks + 1) & 3] + 128 * (ks >> 2));
                     mma_bf16_16816(sb, a0, a1, a2, a3, qb[ks + 1][0], qb[ks + 1][1]);
                 }
 
-                if (it > 0) emit_previous(base);      // the old logits of these slots, before they are overwritten
+                if (it > 0) {      // the previous unit's logits of these slots, before they are overwritten
+                    float y00, y01, y10, y11;
+                    load_logits(j, y00, y01, y10, y11);
+                    emit_previous(base, y00, y01, y10, y11);
+                }
 
                 // scale to the log2 domain, mask the slots past n, keep the logits for the next pass
-                const bool in0 = tok0 + base + g < p.n, in1 = tok0 + base + g + 8 < p.n;
-                const float x00 = in0 ? (sa[0] + sb[0]) * p.scale_log2 : -INFINITY;     // token g,     head h0
-                const float x01 = in0 ? (sa[1] + sb[1]) * p.scale_log2 : -INFINITY;     // token g,     head h1
-                const float x10 = in1 ? (sa[2] + sb[2]) * p.scale_log2 : -INFINITY;     // token g + 8, head h0
-                const float x11 = in1 ? (sa[3] + sb[3]) * p.scale_log2 : -INFINITY;     // token g + 8, head h1
-                if (h0_on) {
-                    logits[h0 * LS + base + g] = x00;
-                    logits[h0 * LS + base + g + 8] = x10;
+                float x00 = (sa[0] + sb[0]) * p.scale_log2;      // token g,     head h0
+                float x01 = (sa[1] + sb[1]) * p.scale_log2;      // token g,     head h1
+                float x10 = (sa[2] + sb[2]) * p.scale_log2;      // token g + 8, head h0
+                float x11 = (sa[3] + sb[3]) * p.scale_log2;      // token g + 8, head h1
+                if (tok0 + base + 16 > p.n) {                    // only the unit's last page can be ragged
+                    if (tok0 + base + g >= p.n) x00 = x01 = -INFINITY;
+                    if (tok0 + base + g + 8 >= p.n) x10 = x11 = -INFINITY;
                 }
-                if (h1_on) {
-                    logits[h1 * LS + base + g] = x01;
-                    logits[h1 * LS + base + g + 8] = x11;
-                }
+                store_logits(j, x00, x01, x10, x11);
 
                 // raise the reference only when some logit is more than 2^8 above it (always on the first tile)
                 float mx0 = fmaxf(x00, x10), mx1 = fmaxf(x01, x11);
@@ -331,15 +392,29 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) {
                     uint32_t a0, a1, a2, a3;
-                    ldmatrix_x4_trans(a0, a1, a2, a3, pb_addr + v_lane + (((2 * mt + v_sel) ^ lrow) << 4));
+                    ldmatrix_x4_trans(a0, a1, a2, a3, page + v_off[mt & 3] + 128 * (mt >> 2));
                     mma_bf16_16816(o[mt], a0, a1, a2, a3, bh0, bh1);
                     mma_bf16_16816(o[mt], a0, a1, a2, a3, bl0, bl1);
                 }
                 // Before the page goes back, look at the barriers of the other groups' pages up to this
                 // group's next one: the producer cannot reuse their stages while this one is held.
                 if (NG > 1) observe_through(pc + NG - 1);
+                if (j < tmem_pages) tmem_wait_st();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[stage]);
+                stage += NG;
+                if (stage >= (uint32_t)NS) {
+                    stage -= NS;
+                    parity ^= 1;
+                }
+            }
+            // ring position of the next unit's first page
+            pc_base += npg;
+            pc_mod = (pc_mod + npg) % NG;
+            {
+                const uint32_t adv = st_base + (uint32_t)npg;
+                par_base ^= (adv / NS) & 1;
+                st_base = adv % NS;
             }
 
             // ---- merge the warps of this block ---------------------------------
@@ -442,13 +517,21 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 
         // probabilities and statistics of the block's last unit
         if (it > 0) {
-            for (int j = 0; j < npg; ++j)
-                if (NG == 1 || j % NG == grp) emit_previous(j * kPageTokens + (int)tok_off);
+            for (int j = grp; j < npg; j += NG) {
+                float y00, y01, y10, y11;
+                load_logits(j, y00, y01, y10, y11);
+                emit_previous(j * kPageTokens + (int)tok_off, y00, y01, y10, y11);
+            }
         }
     }
 
-    // No block may exit while a peer can still read its shared memory.
+    // No block may exit while a peer can still read its shared memory; tensor memory goes back last.
+    tmem_fence_before_sync();
     __syncthreads();
+    if (warp == 0) {
+        tmem_fence_after_sync();
+        tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    }
     if (clustered) {
         cluster_arrive();
         cluster_wait();
@@ -456,6 +539,8 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 }
 
 constexpr int kMaxGroups = 2;
+constexpr int kTmemPages = 128;            // 512 columns / 4 per page
+constexpr size_t kMinSmemBytes = 120 * 1024;
 
 template <int NG>
 cudaError_t launch_impl(const DecodeParams& p, const DecodePlan& plan, int clusters, cudaStream_t stream,
@@ -481,11 +566,17 @@ cudaError_t launch_impl(const DecodeParams& p, const DecodePlan& plan, int clust
 // Shared-memory layout for a given cluster size and ring depth; returns the total bytes.
 static size_t layout(const DecodeConfig& c, int np, int s, int ns, DecodePlan* plan) {
     const int ppc = (np + s - 1) / s;
-    const int ls = ppc * kPageTokens + 4;      // = 4 (mod 32) floats: the rows of a lane's two heads and of the four
-                                               // lanes of a fragment row fall into different banks
+    // Logits live in tensor memory, four columns per page and lane (128 pages at most); the pages
+    // beyond that spill to shared memory, one row per head with a stride = 4 (mod 32) floats, so
+    // that the rows of a lane's two heads and of the four lanes of a fragment row fall into
+    // different banks.
+    const int tp = ppc < kTmemPages ? ppc : kTmemPages;
+    int cols = 32;
+    while (cols < 4 * tp) cols *= 2;
+    const int ls = (ppc - tp) * kPageTokens + 4;
     size_t off = (size_t)ns * kPageBytes;
     plan->off_logits = (int)off;
-    off += ((size_t)c.group * ls * sizeof(float) + 127) / 128 * 128;
+    if (ppc > tp) off += ((size_t)c.group * ls * sizeof(float) + 127) / 128 * 128;
     plan->off_xchg = (int)off;
     off += 2 * sizeof(Xchg);
     plan->off_wml = (int)off;
@@ -499,6 +590,11 @@ static size_t layout(const DecodeConfig& c, int np, int s, int ns, DecodePlan* p
     plan->groups = c.force_groups > 0 ? c.force_groups : 2;
     plan->pages_per_cta = ppc;
     plan->logit_stride = ls;
+    plan->tmem_pages = tp;
+    plan->tmem_cols = cols;
+    // More than half of an SM's shared memory: one block per SM, so the tensor-memory allocation
+    // of one block never waits for another block's.
+    if (off < kMinSmemBytes) off = kMinSmemBytes;
     plan->smem_bytes = (int)off;
     return off;
 }
@@ -551,6 +647,8 @@ cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clu
     p.stages = plan.stages;
     p.pages_per_cta = plan.pages_per_cta;
     p.logit_stride = plan.logit_stride;
+    p.tmem_pages = plan.tmem_pages;
+    p.tmem_cols = plan.tmem_cols;
     p.off_logits = plan.off_logits;
     p.off_xchg = plan.off_xchg;
     p.off_wml = plan.off_wml;

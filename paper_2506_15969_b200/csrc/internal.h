@@ -15,7 +15,7 @@ struct DecodeConfig {
 };
 
 struct DecodePlan {
-    int splits, stages, groups, pages_per_cta, logit_stride;
+    int splits, stages, groups, pages_per_cta, logit_stride, tmem_pages, tmem_cols;
     int off_logits, off_xchg, off_wml, off_misc, off_bars, smem_bytes;
 };
 
