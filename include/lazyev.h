@@ -186,6 +186,8 @@ typedef struct lazyev_info {
     int splits;          /* blocks per unit used by the last decode launch   */
     int stages;          /* pipeline stages used by the last decode launch   */
     int groups;          /* consumer warp groups used by the last decode launch */
+    int tail_units;      /* units of a partly filled last round, given to a second launch (0 = none) */
+    int tail_splits;     /* blocks per unit in that second launch                  */
     int grid;            /* blocks launched by the last decode launch        */
     int smem_bytes;      /* dynamic shared memory of the last decode launch  */
     long long launches;  /* kernels launched by this handle so far           */

@@ -23,7 +23,7 @@ class Info(C.Structure):
     _fields_ = [(n, C.c_int) for n in (
         "layers", "batch", "q_heads", "kv_heads", "head_dim", "units", "budget", "budget_now", "window",
         "n_recent", "n_initial", "capacity", "pages_per_unit", "t", "n", "prefill", "splits", "stages",
-        "groups", "grid", "smem_bytes")] + [("launches", C.c_longlong), ("evictions", C.c_longlong)]
+        "groups", "tail_units", "tail_splits", "grid", "smem_bytes")] + [("launches", C.c_longlong), ("evictions", C.c_longlong)]
 
 
 class Profile(C.Structure):

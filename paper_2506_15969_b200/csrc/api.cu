@@ -38,9 +38,9 @@ struct lazyev {
     int t = 0, n = 0, prefill = 0;
     long long launches = 0, evictions = 0;
     DecodePlan last_plan = {};
-    int last_grid = 0;
+    int last_grid = 0, last_tail_units = 0, last_tail_splits = 0;
     struct Shape {
-        int splits = 1, clusters = 1, forced_splits = 0, forced_stages = 0, forced_groups = 0;
+        int splits = 1, clusters = 1, tail_splits = 0, tail_units = 0, forced_splits = 0, forced_stages = 0, forced_groups = 0;
     };
     std::map<int, Shape> plan_cache;                       // pages in use -> launch shape
     // optional per-kernel timing with CUDA events
@@ -248,9 +248,11 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
 
     DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages, h->force_groups};
-    // Launch shape: among the cluster sizes whose logits fit in shared memory, take the one that keeps
-    // the most SMs busy, discounted when the page ring gets shallow.  The choice depends only on the
-    // number of pages in use, so it is cached per page count.
+    // Launch shape, chosen per number of pages in use and cached.  Every cluster size whose logits fit
+    // gets a relative speed (blocks per unit, discounted for the per-unit exchange between the blocks
+    // of a cluster and for a shallow page ring); the main launch is the size with the least time over
+    // the rounds of the round-robin walk.  A partly filled last round goes to a second launch with
+    // larger clusters when that is faster, so that more SMs share its units.
     const int np = (n + kPageTokens - 1) / kPageTokens;
     auto cached = h->plan_cache.find(np);
     if (cached == h->plan_cache.end() || cached->second.forced_splits != h->force_splits ||
@@ -259,10 +261,12 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
         best.forced_splits = h->force_splits;
         best.forced_stages = h->force_stages;
         best.forced_groups = h->force_groups;
-        double best_score = -1.0;
-        static const double kRingWeight[7] = {0, 0, 0.70, 0.92, 0.97, 1.0, 1.0};
+        // relative speed of one block by ring depth and by cluster size (measured on B200 at 8 k tokens)
+        static const double kRingWeight[7] = {0, 0, 0.70, 0.90, 0.96, 0.99, 1.0};
+        static const double kSplitWeight[9] = {0, 1.0, 0.94, 0.92, 0.90, 0.88, 0.86, 0.84, 0.82};
+        int max_clusters[9] = {0};
+        double speed[9] = {0};                       // units per unit of time done by one cluster of s blocks
         for (int s = 1; s <= 8; ++s) {
-            if (h->force_splits > 0 && s != h->force_splits) continue;
             if (h->force_splits == 0 && s > 1 && (np < 2 * s)) continue;       // at least two pages per block
             DecodePlan plan;
             if (decode_plan(c, n + kPageTokens, h->max_smem, s, &plan) != 0) continue;   // room for the page count to grow by one
@@ -272,35 +276,63 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
                 cudaGetLastError();
                 continue;
             }
-            if (clusters < 1) continue;
-            const int used = clusters < h->units ? clusters : h->units;
-            // rounds of the round-robin walk over units decide the tail: count whole rounds
-            const int rounds = (h->units + used - 1) / used;
-            const double busy = (double)h->units * s / ((double)rounds * h->num_sms);
-            const double score = busy * kRingWeight[plan.stages];
-            if (score > best_score + 1e-9) {
-                best_score = score;
+            max_clusters[s] = clusters;
+            speed[s] = s * kRingWeight[plan.stages] * kSplitWeight[s];
+        }
+        double best_time = -1.0;
+        for (int s = 1; s <= 8; ++s) {
+            if (max_clusters[s] < 1 || (h->force_splits > 0 && s != h->force_splits)) continue;
+            const int used = max_clusters[s] < h->units ? max_clusters[s] : h->units;
+            const int full = h->units / used, rem = h->units % used;
+            double time = full / speed[s];
+            int ts = 0;
+            if (rem > 0) {
+                double tail = 1.0 / speed[s];
+                if (full > 0 && h->force_splits == 0)
+                    for (int k = s + 1; k <= 8; ++k)
+                        if (max_clusters[k] >= rem && rem * k <= h->num_sms && 1.0 / speed[k] < tail) {
+                            tail = 1.0 / speed[k];
+                            ts = k;
+                        }
+                time += tail;
+            }
+            if (best_time < 0 || time < best_time - 1e-12) {
+                best_time = time;
                 best.splits = s;
                 best.clusters = used;
+                best.tail_splits = ts;
+                best.tail_units = ts > 0 ? rem : 0;
             }
         }
-        if (best_score < 0) return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
+        if (best_time < 0) return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
         cached = h->plan_cache.insert_or_assign(np, best).first;
     }
+    const lazyev::Shape shape = cached->second;
     DecodePlan plan;
-    if (decode_plan(c, n, h->max_smem, cached->second.splits, &plan) != 0)
+    if (decode_plan(c, n, h->max_smem, shape.splits, &plan) != 0)
         return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
-    const int clusters = cached->second.clusters;
-    DecodeArgs a{h->pool, h->st, q, out, n, t};
+    DecodePlan tail_plan = {};
+    if (shape.tail_units > 0 && decode_plan(c, n, h->max_smem, shape.tail_splits, &tail_plan) != 0)
+        return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
+    const int main_units = h->units - shape.tail_units;
+    const int clusters = shape.clusters < main_units ? shape.clusters : main_units;
     {
         // algorithmic bytes: every cached K and V row read once, one probability written per token,
         // the queries read and the outputs written
         SpanGuard g(h, kSpanDecode, (double)h->units * ((double)n * (2 * kRowBytes + 4) + 2.0 * h->group * kRowBytes));
+        DecodeArgs a{h->pool, h->st, q, out, n, t, 0, main_units};
         e = decode_launch(c, plan, clusters, a, h->stream);
+        if (e == cudaSuccess && shape.tail_units > 0) {
+            DecodeArgs b{h->pool, h->st, q, out, n, t, main_units, shape.tail_units};
+            e = decode_launch(c, tail_plan, shape.tail_units, b, h->stream);
+            h->launches += 1;
+        }
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "decode kernel launch");
     h->launches += 2;
     h->last_plan = plan;
+    h->last_tail_units = shape.tail_units;
+    h->last_tail_splits = shape.tail_splits;
     h->last_grid = clusters * plan.splits;
     h->t = t;
     h->n = n;
@@ -616,6 +648,8 @@ int lazyev_get_info(const lazyev_t* h, lazyev_info_t* out) {
     out->splits = h->last_plan.splits;
     out->stages = h->last_plan.stages;
     out->groups = h->last_plan.groups;
+    out->tail_units = h->last_tail_units;
+    out->tail_splits = h->last_tail_splits;
     out->grid = h->last_grid;
     out->smem_bytes = h->last_plan.smem_bytes;
     out->launches = h->launches;

@@ -22,8 +22,9 @@
 // that is raised (and O, l rescaled) only when a logit exceeds it by more than
 // 2^8, found with one warp vote per tile; any reference gives the same sums.
 //
-// The scaled logits of the block's chunk stay in shared memory (one float per
-// head and token).  After the chunk the warps and then the cluster's blocks
+// The scaled logits of the block's chunk stay on chip: in tensor memory (TMEM,
+// used as 512 private 32-bit words per consumer thread through tcgen05.ld / st),
+// and in shared memory for the pages beyond the 128 that fit there.  After the chunk the warps and then the cluster's blocks
 // merge (reference, l, O) through (distributed) shared memory, which gives the
 // exact log-sum-exp.  The probabilities of a unit are produced while the block's
 // NEXT unit streams: the warp that is about to overwrite the logits of a
@@ -53,7 +54,7 @@ struct DecodeParams {
     int32_t* ts;
     int32_t* mri;
     int32_t* status;
-    int units, group, pages_per_unit, capacity, total_pages;
+    int unit_begin, unit_end, group, pages_per_unit, capacity, total_pages;     // this launch walks units [begin, end)
     int n, t;
     float alpha, scale_log2, inv_group;
     int splits, stages, pages_per_cta, logit_stride, tmem_pages, tmem_cols;
@@ -141,13 +142,14 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
     const int pg0 = min(np, (int)rank * p.pages_per_cta);
     const int pg1 = min(np, pg0 + p.pages_per_cta);
     const int npg = pg1 - pg0;
-    const int my_units = cluster_id < p.units ? (p.units - cluster_id + n_clusters - 1) / n_clusters : 0;
+    const int n_units = p.unit_end - p.unit_begin;
+    const int my_units = cluster_id < n_units ? (n_units - cluster_id + n_clusters - 1) / n_clusters : 0;
 
     if (warp == NW) {
         // ------------------------------------------------------------ producer
         uint32_t pc = 0, stage = 0, parity = 1;     // parity of the "empty" phase that frees the stage
         int it = 0;
-        for (int u = cluster_id; u < p.units; u += n_clusters, ++it) {
+        for (int u = p.unit_begin + cluster_id; u < p.unit_end; u += n_clusters, ++it) {
             const int32_t* pt = p.page_table + (size_t)u * p.pages_per_unit + pg0;
             for (int base = 0; base < npg; base += 32) {
                 const int cnt = min(32, npg - base);
@@ -216,7 +218,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         const int tok0 = pg0 * kPageTokens;           // first token of this block's chunk
         uint32_t pc_base = 0;                         // pages of this block before the current unit
         uint32_t pc_mod = 0;                          // pc_base mod NG
-        uint32_t st_base = 0, par_base = 0;           // ring stage and "full" parity of page pc_base
+        uint32_t st_base = 0;                         // ring stage of page pc_base
         uint32_t pc_seen = 0, st_seen = 0, par_seen = 0;   // next page whose "full" phase this warp observes
         float lse0 = 0.f, lse1 = 0.f;                 // log-sum-exp of the previous unit, heads h0 and h1
         int u_prev = -1;
@@ -294,7 +296,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
             }
         };
 
-        for (int u = cluster_id; u < p.units; u += n_clusters, ++it) {
+        for (int u = p.unit_begin + cluster_id; u < p.unit_end; u += n_clusters, ++it) {
             // Q^T as the B operand: b0 = Q[head g][16 ks + 2 qd, +1], b1 = the same 8 dims further
             uint32_t qb[8][2];
             {
@@ -312,11 +314,8 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 
             // this group's pages of the unit: j = j0, j0 + NG, ...
             const int j0 = NG == 1 ? 0 : (int)((grp + NG - pc_mod) % NG);
-            uint32_t stage = st_base + j0, parity = par_base;
-            if (stage >= (uint32_t)NS) {
-                stage -= NS;
-                parity ^= 1;
-            }
+            uint32_t stage = st_base + j0;
+            if (stage >= (uint32_t)NS) stage -= NS;
             for (int j = j0; j < npg; j += NG) {
                 const uint32_t pc = pc_base + j;
                 observe_through(pc);
@@ -403,19 +402,12 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&empty[stage]);
                 stage += NG;
-                if (stage >= (uint32_t)NS) {
-                    stage -= NS;
-                    parity ^= 1;
-                }
+                if (stage >= (uint32_t)NS) stage -= NS;
             }
             // ring position of the next unit's first page
             pc_base += npg;
             pc_mod = (pc_mod + npg) % NG;
-            {
-                const uint32_t adv = st_base + (uint32_t)npg;
-                par_base ^= (adv / NS) & 1;
-                st_base = adv % NS;
-            }
+            st_base = (st_base + (uint32_t)npg) % NS;
 
             // ---- merge the warps of this block ---------------------------------
 #pragma unroll
@@ -633,7 +625,8 @@ cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clu
     p.ts = a.state.ts;
     p.mri = a.state.mri;
     p.status = a.state.status;
-    p.units = c.units;
+    p.unit_begin = a.unit_begin;
+    p.unit_end = a.unit_begin + a.unit_count;
     p.group = c.group;
     p.pages_per_unit = c.pages_per_unit;
     p.capacity = c.capacity;

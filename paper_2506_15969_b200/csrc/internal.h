@@ -26,6 +26,7 @@ struct DecodeArgs {
     void* out;
     int n;                 // cached tokens per unit, the new one included
     int t;                 // this decode step
+    int unit_begin, unit_count;   // the units this launch covers
 };
 
 // Deepest ring and the shared-memory layout for n cached tokens and a cluster of `splits` blocks;

@@ -212,9 +212,19 @@ class TraceGen:
     def kv_at(self, pos: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
         """bf16 K and V [U, len(pos), D] of the tokens at the given positions."""
         pos = pos.to(self.device, torch.int64)
-        k = self._normal_int(_ST_K, self.units[:, None], pos[None, :])
-        v = self._normal_int(_ST_V, self.units[:, None], pos[None, :])
-        return self._to_bf16(k), self._to_bf16(v)
+        npos = int(pos.numel())
+        rows = max(1, (1 << 25) // max(1, npos * self.D))       # units per slice: bounds the int64 temporaries
+        if rows >= self.U:
+            k = self._normal_int(_ST_K, self.units[:, None], pos[None, :])
+            v = self._normal_int(_ST_V, self.units[:, None], pos[None, :])
+            return self._to_bf16(k), self._to_bf16(v)
+        k = torch.empty(self.U, npos, self.D, dtype=torch.bfloat16, device=self.device)
+        v = torch.empty_like(k)
+        for a in range(0, self.U, rows):
+            u = self.units[a:a + rows, None]
+            k[a:a + rows] = self._to_bf16(self._normal_int(_ST_K, u, pos[None, :]))
+            v[a:a + rows] = self._to_bf16(self._normal_int(_ST_V, u, pos[None, :]))
+        return k, v
 
     def prefill(self) -> Tuple[torch.Tensor, torch.Tensor]:
         return self.kv_at(torch.arange(self.cfg.prefill, device=self.device))

@@ -34,6 +34,19 @@ def test_attention_and_tracking_without_eviction(splits):
     assert ls.eng.info().splits == splits
 
 
+def test_partly_filled_last_round_goes_to_a_second_launch():
+    """158 units on 148 SMs: 148 in the main launch, the other 10 in a launch with larger clusters."""
+    cfg = traces.tiny_config(batch=2, layers=79, q_heads=7, kv_heads=1, budget=300, window=32, prefill=280)
+    ls = lockstep(cfg, seed=14, sample_units=[0, 1, 147, 148, 149, 156, 157], pure=False)
+    ls.run(40)
+    ls.assert_ok()
+    inf = ls.eng.info()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert inf.splits == 1 and inf.grid == sms
+    assert inf.tail_units == cfg.units - sms and inf.tail_splits > 1
+    assert ls.rep.evictions == 1
+
+
 def test_softmax_reference_is_raised_late():
     """Logits that grow by far more than the 2^8 margin inside one unit, and a dominant token:
     the lazily raised softmax reference must give the same sums as an exact running maximum."""
