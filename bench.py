@@ -194,22 +194,17 @@ def run_reference(args):
 # ------------------------------------------------------------------ the CUDA leg
 def run_ours(args):
     import torch
-    from paper_2506_15969_b200 import binding, traces
+    from paper_2506_15969_b200 import binding, replicas, traces
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = replicas.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dist = replicas.init("nccl", torch.device("cuda", local))
 
     cfg = pick_config(args)
     # every rank runs the same per-GPU workload on its own replica of the batch (weak scaling, no exchange)
-    gen = traces.TraceGen(cfg, args.seed + 1000 * rank, device="cuda")
+    gen = traces.TraceGen(cfg, replicas.replica_seed(args.seed, rank), device="cuda")
     eng = binding.Engine(cfg.layers, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window,
                          cfg.threshold, batch=cfg.batch, n_recent=cfg.n_recent, n_initial=cfg.n_initial,
                          max_prefill=cfg.prefill)
@@ -267,10 +262,7 @@ def run_ours(args):
     eng.synchronize()
 
     def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier(dist, torch.cuda.synchronize)
 
     # ---- headline: K steps, inputs resident in HBM, device-timed -------------------
     sampler = ClockSampler(local)
@@ -283,12 +275,9 @@ def run_ours(args):
     sampler.join(timeout=2)
     launches = eng.info().launches - launches0
     evictions_timed = sum(1 for x in range(t_first, t + 1) if x % cfg.window == 0)
-    if dist is not None:
-        tmax = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = replicas.max_over_ranks(ms, dist, "cuda")
     inf = eng.info()
-    value = world * cfg.batch * args.steps / (ms * 1e-3)
+    value = replicas.job_tokens_per_second(cfg.batch, args.steps, world, ms)
 
     # ---- per-kernel roofline: one observation window with events around each kernel ----
     roofline, kernels = None, None
@@ -323,13 +312,10 @@ def run_ours(args):
         barrier()
         wall_ms = run_steps(e2e_steps, host=True)
         barrier()
-        if dist is not None:
-            tmax = torch.tensor([wall_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            wall_ms = float(tmax.item())
+        wall_ms = replicas.max_over_ranks(wall_ms, dist, "cuda")
         qbytes = L * Bt * cfg.q_heads * cfg.head_dim * 2
         kbytes = L * Bt * cfg.kv_heads * cfg.head_dim * 2
-        e2e = {"value": world * cfg.batch * e2e_steps / (wall_ms * 1e-3), "unit": "tokens/s",
+        e2e = {"value": replicas.job_tokens_per_second(cfg.batch, e2e_steps, world, wall_ms), "unit": "tokens/s",
                "h2d_bytes_per_step": qbytes + 2 * kbytes, "d2h_bytes_per_step": qbytes, "steps": e2e_steps,
                "ms_per_step": wall_ms / e2e_steps}
     eng.synchronize()
