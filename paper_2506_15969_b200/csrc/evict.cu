@@ -31,40 +31,28 @@ __device__ __forceinline__ double score_fn(int d, int mri, int mode) {
 
 constexpr int kSelThreads = 512;
 
-// Exclusive prefix sum of one int per thread over the block; *total gets the block sum.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
+// Block-wide sum of one int per thread.
+__device__ __forceinline__ int block_sum(int v, int* warp_sums) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int inc = v;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int up = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += up;
-    }
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     __syncthreads();                       // warp_sums may still be read from a previous call
-    if (lane == 31) warp_sums[warp] = inc;
+    if (lane == 0) warp_sums[warp] = v;
     __syncthreads();
-    if (warp == 0) {
-        int s = lane < kSelThreads / 32 ? warp_sums[lane] : 0;
+    int s = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, s, o);
-            if (lane >= o) s += up;
-        }
-        if (lane < kSelThreads / 32) warp_sums[lane] = s;      // inclusive sums of the warps
-    }
-    __syncthreads();
-    *total = warp_sums[kSelThreads / 32 - 1];
-    return inc - v + (warp > 0 ? warp_sums[warp - 1] : 0);
+    for (int w = 0; w < kSelThreads / 32; ++w) s += warp_sums[w];
+    return s;
 }
 
 __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, StateView st, EvictArgs a) {
     extern __shared__ __align__(16) unsigned long long keys[];
     __shared__ unsigned int hist[256];
     __shared__ unsigned long long sh_prefix;
-    __shared__ int sh_krem, sh_first;
+    __shared__ int sh_krem, sh_first, sh_done;
     __shared__ int warp_sums[kSelThreads / 32];
 
-    const int u = blockIdx.x, tid = threadIdx.x;
+    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int S = a.n_initial, R = a.n_recent;
     const int ncand = a.n - R - S;                 // unprotected slots [S, n - R)
     const int k = a.budget - R - S;                // how many of them stay
@@ -72,75 +60,129 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     const int32_t* mri = st.mri + (size_t)u * geo.capacity + S;
     int32_t* src = a.src + (size_t)u * a.budget;
 
-    for (int i = tid; i < ncand; i += kSelThreads)
-        keys[i] = (unsigned long long)__double_as_longlong(score_fn(a.t - ts[i], mri[i], a.score_mode));
-    if (tid == 0) sh_first = ncand;
-    __syncthreads();
-
-    // Radix select, most significant byte first: the bit pattern of the k-th largest score.
-    // Scores are >= 0, so their IEEE bit patterns order like unsigned integers.
-    unsigned long long prefix = 0, mask = 0;
-    int krem = k;
-    for (int shift = 56; shift >= 0; shift -= 8) {
-        if (tid < 256) hist[tid] = 0;
-        __syncthreads();
-        for (int i = tid; i < ncand; i += kSelThreads) {
-            const unsigned long long key = keys[i];
-            if ((key & mask) == prefix) atomicAdd(&hist[(unsigned)(key >> shift) & 255u], 1u);
-        }
-        __syncthreads();
-        if (tid == 0) {
-            int cum = 0, digit = 0;
-            for (int b = 255; b >= 0; --b) {
-                const int c = (int)hist[b];
-                if (cum + c >= krem) {
-                    digit = b;
-                    break;
-                }
-                cum += c;
-            }
-            sh_prefix = prefix | ((unsigned long long)digit << shift);
-            sh_krem = krem - cum;
-        }
-        __syncthreads();
-        prefix = sh_prefix;
-        krem = sh_krem;
-        mask |= 0xFFull << shift;
+    // Scores are >= 0, so their IEEE bit patterns order like unsigned integers; a score of exactly 0
+    // (never re-activated, the common case) has key 0.
+    int nonzero = 0;
+    for (int i = tid; i < ncand; i += kSelThreads) {
+        const unsigned long long key =
+            (unsigned long long)__double_as_longlong(score_fn(a.t - ts[i], mri[i], a.score_mode));
+        keys[i] = key;
+        nonzero += key != 0ull;
     }
-    const unsigned long long kth = prefix;         // keep every key > kth, and `krem` of the keys == kth
+    if (tid == 0) sh_first = ncand;
+    nonzero = block_sum(nonzero, warp_sums);       // (its barriers also publish keys[] and sh_first)
+
+    // kth: bit pattern of the k-th largest score; krem: how many of the keys equal to it stay.
+    unsigned long long kth = 0;
+    int krem = k - nonzero;
+    if (nonzero > k) {
+        // Radix select over the non-zero keys, most significant byte first.  The histogram is built with
+        // one shared-memory atomic per distinct digit and warp (scores cluster in a few exponents), and
+        // the passes stop as soon as the k-th key is alone in its bin.
+        unsigned long long prefix = 0, mask = 0;
+        krem = k;
+        for (int shift = 56; shift >= 0; shift -= 8) {
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            for (int i0 = 0; i0 < ncand; i0 += kSelThreads) {
+                const int i = i0 + tid;
+                const unsigned long long key = i < ncand ? keys[i] : 0ull;
+                const bool on = key != 0ull && (key & mask) == prefix;
+                const unsigned digit = on ? (unsigned)(key >> shift) & 255u : 256u;
+                const unsigned peers = __match_any_sync(0xffffffffu, digit);
+                if (on && (int)(__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], (unsigned)__popc(peers));
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int cum = 0, digit = 0;
+                for (int b = 255; b >= 0; --b) {
+                    const int c = (int)hist[b];
+                    if (cum + c >= krem) {
+                        digit = b;
+                        break;
+                    }
+                    cum += c;
+                }
+                sh_prefix = prefix | ((unsigned long long)digit << shift);
+                sh_krem = krem - cum;
+                sh_done = hist[digit] == 1u;
+            }
+            __syncthreads();
+            prefix = sh_prefix;
+            krem = sh_krem;
+            mask |= 0xFFull << shift;
+            if (sh_done) break;                    // uniform: read from shared memory after the barrier
+        }
+        kth = prefix;
+        if (mask != ~0ull) {                       // stopped early: the only key with this prefix is the k-th
+            __syncthreads();
+            for (int i = tid; i < ncand; i += kSelThreads)
+                if (keys[i] != 0ull && (keys[i] & mask) == prefix) sh_prefix = keys[i];
+            __syncthreads();
+            kth = sh_prefix;
+        }
+    }
+    // keep every key > kth, and `krem` of the keys == kth
 
     // Ties are resolved towards the more recent token, i.e. the higher slot: keep the last `krem` ties.
-    const int ipt = (ncand + kSelThreads - 1) / kSelThreads;
-    const int b = min(ncand, tid * ipt), e = min(ncand, b + ipt);
+    // Each warp owns a contiguous segment of the candidates and walks it 32 at a time, so ranks in
+    // slot order come from ballots: lanes read consecutive keys (no bank conflicts).
+    constexpr int kWarps = kSelThreads / 32;
+    const int warp = tid >> 5;
+    const int seg = ((ncand + kWarps - 1) / kWarps + 31) / 32 * 32;
+    const int seg_b = min(ncand, warp * seg), seg_e = min(ncand, seg_b + seg);
+    const unsigned lt = (1u << lane) - 1u;
     int ties = 0;
-    for (int i = b; i < e; ++i) ties += keys[i] == kth;
-    int total_ties;
-    int tie_rank = block_exclusive_scan(ties, warp_sums, &total_ties);
+    for (int i0 = seg_b; i0 < seg_e; i0 += 32) {
+        const int i = i0 + lane;
+        ties += __popc(__ballot_sync(0xffffffffu, i < seg_e && keys[i] == kth));
+    }
+    __syncthreads();
+    if (lane == 0) warp_sums[warp] = ties;
+    __syncthreads();
+    int tie_rank = 0, total_ties = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        tie_rank += w < warp ? warp_sums[w] : 0;
+        total_ties += warp_sums[w];
+    }
     const int first_kept_tie = total_ties - krem;
+    unsigned long long keep_bits = 0;              // bit j: this lane's candidate of step j stays (at most 50 steps)
     int kept = 0;
     {
-        int r = tie_rank;
-        for (int i = b; i < e; ++i) {
-            const unsigned long long key = keys[i];
-            bool keep = key > kth;
-            if (key == kth) keep = r++ >= first_kept_tie;
-            kept += keep;
+        int step = 0;
+        for (int i0 = seg_b; i0 < seg_e; i0 += 32, ++step) {
+            const int i = i0 + lane;
+            const unsigned long long key = i < seg_e ? keys[i] : 0ull;
+            const bool tie = i < seg_e && key == kth;
+            const unsigned tie_mask = __ballot_sync(0xffffffffu, tie);
+            const bool keep = i < seg_e && (key > kth || (tie && tie_rank + __popc(tie_mask & lt) >= first_kept_tie));
+            tie_rank += __popc(tie_mask);
+            kept += __popc(__ballot_sync(0xffffffffu, keep));
+            keep_bits |= (unsigned long long)keep << step;
         }
     }
-    int total_kept;
-    int dst = block_exclusive_scan(kept, warp_sums, &total_kept);
+    __syncthreads();
+    if (lane == 0) warp_sums[warp] = kept;
+    __syncthreads();
+    int dst = 0, total_kept = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        dst += w < warp ? warp_sums[w] : 0;
+        total_kept += warp_sums[w];
+    }
     {
-        int r = tie_rank, first_evicted = ncand;
-        for (int i = b; i < e; ++i) {
-            const unsigned long long key = keys[i];
-            bool keep = key > kth;
-            if (key == kth) keep = r++ >= first_kept_tie;
-            if (keep)
-                src[S + dst++] = S + i;
-            else if (first_evicted == ncand)
-                first_evicted = i;
+        int step = 0, first_evicted = ncand;
+        for (int i0 = seg_b; i0 < seg_e; i0 += 32, ++step) {
+            const int i = i0 + lane;
+            const bool keep = (keep_bits >> step) & 1ull;
+            const unsigned keep_mask = __ballot_sync(0xffffffffu, keep);
+            if (keep) src[S + dst + __popc(keep_mask & lt)] = S + i;
+            dst += __popc(keep_mask);
+            const unsigned gone = __ballot_sync(0xffffffffu, i < seg_e && !keep);
+            if (gone != 0u && first_evicted == ncand) first_evicted = i0 + __ffs(gone) - 1;
         }
-        if (first_evicted < ncand) atomicMin(&sh_first, first_evicted);
+        if (lane == 0 && first_evicted < ncand) atomicMin(&sh_first, first_evicted);
     }
     for (int j = tid; j < S; j += kSelThreads) src[j] = j;
     for (int r = tid; r < R; r += kSelThreads) src[a.budget - R + r] = a.n - R + r;
@@ -153,52 +195,65 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
 
 constexpr int kCompactThreads = 256;
 constexpr int kRowsPerWarp = kPageTokens / (kCompactThreads / 32);     // 8
+constexpr int kMaxPagesInSmem = 1024;                                  // page-table entries cached per block
 
 // One block per unit walks destination pages front to back.  Destination slot j
 // receives slot src[j] >= j, and sources are strictly increasing in j, so once a
 // tile's sources sit in registers (barrier) its destinations can be overwritten:
-// they are sources only of this or of earlier tiles.
-__global__ void __launch_bounds__(kCompactThreads) compact_kernel(Geometry geo, uint8_t* pool, StateView st,
+// they are sources only of this or of earlier tiles.  The source indices of the
+// next tile are fetched while the rows of the current one are in flight, and the
+// unit's page table sits in shared memory, so a tile costs one global round trip.
+__global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(Geometry geo, uint8_t* pool, StateView st,
                                                                  EvictArgs a) {
+    __shared__ int32_t pt_s[kMaxPagesInSmem];
     const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int32_t* src = a.src + (size_t)u * a.budget;
-    const int32_t* pt = st.page_table + (size_t)u * geo.pages_per_unit;
+    const int32_t* pt_g = st.page_table + (size_t)u * geo.pages_per_unit;
     const int first = a.first_moved[u];
     const size_t sbase = (size_t)u * geo.capacity;
     const int half = lane < 16 ? 0 : kPageHalfBytes;      // lanes 0..15: K row, 16..31: V row
     const int cp = lane & 15;                             // physical chunk read from the source row
+    const bool pt_cached = geo.pages_per_unit <= kMaxPagesInSmem;
+    if (pt_cached)
+        for (int i = tid; i < geo.pages_per_unit; i += kCompactThreads) pt_s[i] = pt_g[i];
+    __syncthreads();
+    const int32_t* pt = pt_cached ? pt_s : pt_g;
 
-    for (int d0 = first / kPageTokens * kPageTokens; d0 < a.budget; d0 += kPageTokens) {
-        uint4 val[kRowsPerWarp];
-        int srow[kRowsPerWarp];
+    // source slot of destination slot dj, or -1 when the row stays where it is
+    auto source_of = [&](int dj) -> int {
+        if (dj < first || dj >= a.budget) return -1;
+        const int sj = src[dj];
+        return sj != dj ? sj : -1;
+    };
+
+    int d0 = first / kPageTokens * kPageTokens;
+    int srow[kRowsPerWarp], s_from = -1;
 #pragma unroll
-        for (int i = 0; i < kRowsPerWarp; ++i) {
-            const int dj = d0 + warp + 8 * i;
-            srow[i] = -1;
-            if (dj >= first && dj < a.budget) {
-                const int sj = src[dj];
-                if (sj != dj) {
-                    srow[i] = sj;
-                    const uint8_t* row =
-                        page_ptr(pool, pt[sj / kPageTokens]) + half + (sj % kPageTokens) * kRowBytes;
-                    val[i] = *reinterpret_cast<const uint4*>(row + cp * 16);
-                }
+    for (int i = 0; i < kRowsPerWarp; ++i) srow[i] = source_of(d0 + warp + 8 * i);
+    if (tid < kPageTokens) s_from = source_of(d0 + tid);
+
+    for (; d0 < a.budget; d0 += kPageTokens) {
+        uint4 val[kRowsPerWarp];
+#pragma unroll
+        for (int i = 0; i < kRowsPerWarp; ++i)
+            if (srow[i] >= 0) {
+                const uint8_t* row =
+                    page_ptr(pool, pt[srow[i] / kPageTokens]) + half + (srow[i] % kPageTokens) * kRowBytes;
+                val[i] = *reinterpret_cast<const uint4*>(row + cp * 16);
             }
+        int s_ts = 0, s_mri = 0, s_pos = 0;
+        if (s_from >= 0) {
+            s_ts = st.ts[sbase + s_from];
+            s_mri = st.mri[sbase + s_from];
+            s_pos = st.pos[sbase + s_from];
         }
-        int s_ts = 0, s_mri = 0, s_pos = 0, s_from = -1;
-        if (tid < kPageTokens) {
-            const int dj = d0 + tid;
-            if (dj >= first && dj < a.budget) {
-                const int sj = src[dj];
-                if (sj != dj) {
-                    s_from = sj;
-                    s_ts = st.ts[sbase + sj];
-                    s_mri = st.mri[sbase + sj];
-                    s_pos = st.pos[sbase + sj];
-                }
-            }
-        }
-        __syncthreads();
+        // next tile's source indices: in flight together with this tile's rows
+        int srow_next[kRowsPerWarp], s_from_next = -1;
+#pragma unroll
+        for (int i = 0; i < kRowsPerWarp; ++i) srow_next[i] = source_of(d0 + kPageTokens + warp + 8 * i);
+        if (tid < kPageTokens) s_from_next = source_of(d0 + kPageTokens + tid);
+
+        __syncthreads();       // every source row of this tile is in registers
         uint8_t* dpage = page_ptr(pool, pt[d0 / kPageTokens]) + half;
 #pragma unroll
         for (int i = 0; i < kRowsPerWarp; ++i) {
@@ -207,12 +262,14 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(Geometry geo, 
                 const int c = cp ^ (srow[i] & 7);              // logical chunk held by this lane
                 *reinterpret_cast<uint4*>(dpage + dr * kRowBytes + swz_chunk(c, dr) * 16) = val[i];
             }
+            srow[i] = srow_next[i];
         }
         if (s_from >= 0) {
             st.ts[sbase + d0 + tid] = s_ts;
             st.mri[sbase + d0 + tid] = s_mri;
             st.pos[sbase + d0 + tid] = s_pos;
         }
+        s_from = s_from_next;
     }
 }
 
