@@ -35,6 +35,29 @@ if ROOT not in sys.path:
 
 METRIC = "decode tokens/sec (all layers, batch B) and fraction of B200 HBM roofline"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM traffic of the decode kernel from the ncu capture summarised in
+# profiles/decode_kernel_cfg4_small_ncu.md: (dram read + write bytes) / algorithmic bytes on a
+# 592-unit case of the same launch shape; traffic grows in proportion to units x tokens, so a full
+# launch is scaled by its algorithmic bytes.  Valid only for the kernel sources it was taken on.
+NCU_DECODE_CAPTURE = {
+    "traffic_per_algorithmic_byte": 1.0080,
+    "sha256": {"decode.cu": "cdadef6063986bfef98f17ef539659e9af82c5c6d780106325e27dbcf87a0519",
+               "common.cuh": "e145966ccf290b94a07f9b5374ce552520833824b6b9440fc6aa85adf416adac"},
+}
+
+
+def ncu_traffic(bytes_per_launch):
+    """Per-launch DRAM bytes scaled from the committed ncu capture, or None once the kernel changed."""
+    import hashlib
+    csrc = os.path.join(ROOT, "paper_2506_15969_b200", "csrc")
+    for name, want in NCU_DECODE_CAPTURE["sha256"].items():
+        try:
+            with open(os.path.join(csrc, name), "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest() != want:
+                    return None
+        except OSError:
+            return None
+    return NCU_DECODE_CAPTURE["traffic_per_algorithmic_byte"] * bytes_per_launch
 
 
 def parse_args():
@@ -46,6 +69,7 @@ def parse_args():
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch (profiling on small cases)")
+    ap.add_argument("--layers", type=int, default=0, help="override the configuration's layer count (profiling on small cases)")
     ap.add_argument("--start-step", type=int, default=-1,
                     help="decode steps replayed untimed before the timed region (-1: up to the first eviction)")
     ap.add_argument("--fast-start", action="store_true",
@@ -66,6 +90,8 @@ def pick_config(args):
     cfg = traces.CONFIGS[args.config]
     if args.batch:
         cfg = dataclasses.replace(cfg, batch=args.batch, name=f"{cfg.name}-batch{args.batch}")
+    if args.layers:
+        cfg = dataclasses.replace(cfg, layers=args.layers, name=f"{cfg.name}-layers{args.layers}")
     if args.fast_start:
         cfg = dataclasses.replace(cfg, prefill=cfg.budget_at(0) if cfg.budget_frac_tenths else cfg.budget,
                                   name=cfg.name + "-faststart")
@@ -291,7 +317,10 @@ def run_ours(args):
         dec_gbs = pr.decode_bytes / (pr.decode_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "decode_kernel (attention + probabilities + TS/MRI update)",
                     "achieved": round(dec_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
-                    "peak_kind": peak_kind, "frac_of_8TBps_nominal": round(dec_gbs / 8000.0, 4), "traffic": None,
+                    "peak_kind": peak_kind, "frac_of_8TBps_nominal": round(dec_gbs / 8000.0, 4),
+                    "traffic": ncu_traffic(pr.decode_bytes / max(pr.decode_launches, 1)),
+                    "traffic_source": "ncu dram__bytes_read+write on a 592-unit case of the same launch shape, "
+                                      "scaled by algorithmic bytes (null if the kernel changed since)",
                     "ms_per_launch": round(pr.decode_ms / max(pr.decode_launches, 1), 4),
                     "bytes_per_launch": pr.decode_bytes / max(pr.decode_launches, 1)}
         kernels = {"append_ms_per_launch": round(pr.append_ms / max(pr.append_launches, 1), 4)}
@@ -344,6 +373,7 @@ def run_ours(args):
                        "window": cfg.window, "prefill": cfg.prefill, "threshold": cfg.threshold,
                        "l2": "inputs larger than L2 (KV pool %.1f GB streamed once per step)" % (eng.kv_pool.numel() / 1e9),
                        "decode_launch": {"splits": inf.splits, "stages": inf.stages, "groups": inf.groups, "grid": inf.grid,
+                                         "tail_units": inf.tail_units, "tail_splits": inf.tail_splits,
                                          "smem_bytes": inf.smem_bytes},
                        "multi_gpu": "independent replicas of the batch per GPU, no collective"},
             "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),
