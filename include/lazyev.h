@@ -52,7 +52,13 @@ enum {
 
 /* Importance score variants: Eq. (2) of the paper and its two ablations
  * (the rows "w/o H2" and "w/o H1" of the score ablation table). */
-enum { LAZYEV_SCORE_H1_PLUS_H2 = 0, LAZYEV_SCORE_H1_ONLY = 1, LAZYEV_SCORE_H2_ONLY = 2 };
+enum {
+    LAZYEV_SCORE_H1_PLUS_H2 = 0,            /* Eq. (2) as printed */
+    LAZYEV_SCORE_H1_ONLY = 1,               /* ablation: without the H2-score */
+    LAZYEV_SCORE_H2_ONLY = 2,               /* ablation: without the H1-score */
+    LAZYEV_SCORE_H1_PLUS_H2_DECREASING = 3  /* Eq. (2) with H2 = 2 sigma(-(MRI - 1)): falls with MRI, as Section 4's
+                                               prose and the appendix on the score's formulation require */
+};
 
 /*
  * Create a handle.  The seven parameters are the method's: model shape, KV
@@ -217,6 +223,26 @@ typedef struct lazyev_dump {
 } lazyev_dump_t;
 
 int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* dump);
+
+/*
+ * Distribution of the recurrence intervals in the live cache (Section 4, "Discussion about
+ * the choice of W and alpha": the paper sets W to the MRI value below which 80 % of the
+ * tokens fall, found offline).  host_hist[b], b < bins - 1, receives the number of cached
+ * tokens of units [unit_begin, unit_begin + unit_count) whose MRI equals b (b = 0: never
+ * re-activated); host_hist[bins - 1] the number with MRI >= bins - 1.  2 <= bins <= 65536;
+ * host_hist is a host array of `bins` 64-bit counts.  Synchronises the stream.
+ * Errors: EINVAL (range, bins, null), ESTATE (before prefill), ECUDA.
+ */
+int lazyev_mri_histogram(lazyev_t* h, int unit_begin, int unit_count, long long* host_hist, int bins);
+
+/*
+ * The rule above as one call: *value = the smallest v such that at least `fraction` (in
+ * (0, 1]) of the re-activated tokens (MRI >= 1) of the unit range have MRI <= v; 0 when no
+ * token has been re-activated yet.  *recurring (may be NULL) = how many such tokens there are.
+ * Whether the paper's 80 % counts all tokens or only re-activated ones is not stated; counting
+ * only re-activated ones keeps the value meaningful when most tokens never recur.
+ */
+int lazyev_mri_quantile(lazyev_t* h, int unit_begin, int unit_count, double fraction, int* value, long long* recurring);
 
 /*
  * Per-kernel timing for benchmarks.  While profiling is on, every kernel launch

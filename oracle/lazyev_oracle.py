@@ -15,6 +15,8 @@ What it follows (paper sections / equations):
 * importance score ............ Section 4 "MRI-Centric Eviction": H1, H2, Eq. (2).
 * lagged eviction ............. Section 4 first paragraph, Appendix A Eq. (evic),
   Algorithm 1 (the `t == kW` branch).
+* MRI distribution ............ Section 4 "Discussion about the choice of W and alpha"
+  (histogram of MRI and the value below which a given share of the tokens falls).
 
 Readings taken where the paper is silent or inconsistent (each is listed with
 its reason in the design notes of the repository):
@@ -46,7 +48,7 @@ import math
 
 import numpy as np
 
-SCORE_MODES = ("h1+h2", "h1", "h2")
+SCORE_MODES = ("h1+h2", "h1", "h2", "h1+h2dec")
 
 
 def bf16_bits_to_f64(bits) -> np.ndarray:
@@ -90,10 +92,27 @@ def h2_score(mri) -> np.ndarray:
     return out
 
 
+def h2_decreasing(mri) -> np.ndarray:
+    """A variant of H2 that does what the paper's prose asks of it: 2*sigma(-(MRI[i] - 1)).
+
+    Section 4 says that a smaller MRI must score higher, and the appendix on the score's
+    formulation requires a monotonically decreasing function with values in [0, 1]; the
+    printed H2 increases with MRI.  Dropping the reciprocal from the printed argument gives
+    the same 2*sigma(-x) form as H1 with x = MRI - 1 >= 0: 1 at MRI = 1, falling to 0.
+    MRI = 0 stays 0 as in the text.  This is a reading offered as a switch, not the default.
+    """
+    mri = np.asarray(mri, dtype=np.int64)
+    out = np.zeros(mri.shape, dtype=np.float64)
+    on = mri >= 1
+    out[on] = 2.0 * sigmoid(-(mri[on].astype(np.float64) - 1.0))
+    return out
+
+
 def importance(t, ts, mri, mode: str = "h1+h2") -> np.ndarray:
     """I_t[i] of Eq. (2): H1 + H2 when MRI != 0, H1 alone when MRI = 0.
 
-    `mode` selects the paper's ablations: "h1" (without H2), "h2" (without H1).
+    `mode` selects the paper's ablations: "h1" (without H2), "h2" (without H1), and
+    "h1+h2dec", Eq. (2) with the decreasing variant of H2.
     """
     if mode not in SCORE_MODES:
         raise ValueError(f"unknown score mode {mode!r}")
@@ -104,7 +123,35 @@ def importance(t, ts, mri, mode: str = "h1+h2") -> np.ndarray:
         return h1
     if mode == "h2":
         return h2
+    if mode == "h1+h2dec":
+        return h1 + np.where(mri != 0, h2_decreasing(mri), 0.0)
     return h1 + h2
+
+
+def mri_histogram(mri_arrays, bins: int) -> np.ndarray:
+    """Counts of MRI values over the cached tokens of several units: out[b] = tokens with
+    MRI = b for b < bins - 1, out[bins - 1] = tokens with MRI >= bins - 1."""
+    out = np.zeros(bins, dtype=np.int64)
+    for arr in mri_arrays:
+        for v in np.asarray(arr, dtype=np.int64):
+            out[min(int(v), bins - 1)] += 1
+    return out
+
+
+def mri_quantile(mri_arrays, fraction: float):
+    """The paper's rule for the observation window (Section 4, "Discussion about the choice
+    of W and alpha": W = the MRI value below which 80 % of the tokens fall), over the
+    re-activated tokens (MRI >= 1): the smallest v with #(MRI <= v) >= fraction * #(MRI >= 1).
+    Returns (v, number of re-activated tokens); v = 0 when there are none."""
+    vals = np.sort(np.concatenate([np.asarray(a, dtype=np.int64) for a in mri_arrays]))
+    vals = vals[vals >= 1]
+    if vals.size == 0:
+        return 0, 0
+    need = fraction * vals.size
+    for rank, v in enumerate(vals, start=1):
+        if rank >= need:
+            return int(v), int(vals.size)
+    return int(vals[-1]), int(vals.size)
 
 
 def attention(q, K, V):

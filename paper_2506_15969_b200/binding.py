@@ -16,7 +16,7 @@ import numpy as np
 from . import build as _build
 
 OK, EINVAL, ESTATE, ECAPACITY, EDEVICE, ECUDA = 0, -1, -2, -3, -4, -5
-SCORE_H1_PLUS_H2, SCORE_H1_ONLY, SCORE_H2_ONLY = 0, 1, 2
+SCORE_H1_PLUS_H2, SCORE_H1_ONLY, SCORE_H2_ONLY, SCORE_H1_PLUS_H2_DECREASING = 0, 1, 2, 3
 
 
 class Info(C.Structure):
@@ -61,6 +61,8 @@ _PROTOS = {
     "lazyev_evict_static": [C.c_void_p, C.POINTER(C.c_int)],
     "lazyev_get_info": [C.c_void_p, C.POINTER(Info)],
     "lazyev_dump_state": [C.c_void_p, C.POINTER(Dump)],
+    "lazyev_mri_histogram": [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int],
+    "lazyev_mri_quantile": [C.c_void_p, C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int), C.POINTER(C.c_longlong)],
     "lazyev_set_profiling": [C.c_void_p, C.c_int],
     "lazyev_get_profile": [C.c_void_p, C.POINTER(Profile), C.c_int],
     "lazyev_synchronize": [C.c_void_p],
@@ -188,6 +190,20 @@ class Engine:
         n = C.c_int()
         self._check(lib().lazyev_evict_static(self._h, C.byref(n)))
         return n.value
+
+    def mri_histogram(self, bins: int, unit_begin: int = 0, unit_count: Optional[int] = None):
+        """lazyev_mri_histogram: int64 counts per MRI value (last bin: everything larger)."""
+        cnt = self.info().units - unit_begin if unit_count is None else unit_count
+        hist = np.zeros(bins, dtype=np.int64)
+        self._check(lib().lazyev_mri_histogram(self._h, unit_begin, cnt, hist.ctypes.data, bins))
+        return hist
+
+    def mri_quantile(self, fraction: float, unit_begin: int = 0, unit_count: Optional[int] = None):
+        """lazyev_mri_quantile: (value, number of re-activated tokens)."""
+        cnt = self.info().units - unit_begin if unit_count is None else unit_count
+        value, total = C.c_int(), C.c_longlong()
+        self._check(lib().lazyev_mri_quantile(self._h, unit_begin, cnt, fraction, C.byref(value), C.byref(total)))
+        return value.value, total.value
 
     def synchronize(self) -> None:
         self._check(lib().lazyev_synchronize(self._h))

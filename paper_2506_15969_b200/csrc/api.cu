@@ -34,6 +34,7 @@ struct lazyev {
     uint8_t* stage_v = nullptr;
     uint8_t* stage_out = nullptr;
     double* stage_score = nullptr;
+    unsigned long long* stage_hist = nullptr;
     // progress
     int t = 0, n = 0, prefill = 0;
     long long launches = 0, evictions = 0;
@@ -59,6 +60,7 @@ struct lazyev {
 namespace {
 
 constexpr int kScoreStageUnits = 32;      // units whose scores one dump pass evaluates
+constexpr int kMaxHistBins = 1 << 16;     // bins of lazyev_mri_histogram()
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -87,7 +89,7 @@ void derive(lazyev_t* h) {
 struct Sizes {
     size_t kv, state, scratch;
     size_t off_ts, off_mri, off_pos, off_pbar, off_status;                          // inside state
-    size_t off_first, off_q, off_k, off_v, off_out, off_score;                      // inside scratch
+    size_t off_first, off_q, off_k, off_v, off_out, off_score, off_hist;            // inside scratch
 };
 
 Sizes sizes_of(const lazyev_t* h) {
@@ -121,6 +123,8 @@ Sizes sizes_of(const lazyev_t* h) {
     off += align_up(qbytes, 256);
     s.off_score = off;
     off += align_up((size_t)kScoreStageUnits * h->capacity * sizeof(double), 256);
+    s.off_hist = off;
+    off += align_up((size_t)kMaxHistBins * sizeof(unsigned long long), 256);
     s.scratch = off;
     return s;
 }
@@ -426,7 +430,7 @@ int lazyev_set_auto_evict(lazyev_t* h, int on) {
 
 int lazyev_set_score_mode(lazyev_t* h, int mode) {
     if (!h) return LAZYEV_EINVAL;
-    if (mode < 0 || mode > 2) return fail(h, LAZYEV_EINVAL, "unknown score mode %d", mode);
+    if (mode < 0 || mode > 3) return fail(h, LAZYEV_EINVAL, "unknown score mode %d", mode);
     h->score_mode = mode;
     return LAZYEV_OK;
 }
@@ -496,6 +500,7 @@ int lazyev_bind(lazyev_t* h, void* kv_pool, void* state, void* scratch, void* cu
     h->stage_v = cp + s.off_v;
     h->stage_out = cp + s.off_out;
     h->stage_score = (double*)(cp + s.off_score);
+    h->stage_hist = (unsigned long long*)(cp + s.off_hist);
 
     // Slots past n are read (and masked) by the decode kernel's last page: they must hold finite values.
     e = cudaMemsetAsync(h->pool, 0, s.kv, h->stream);
@@ -715,6 +720,44 @@ int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* d) {
     if (e != cudaSuccess) return cuda_fail(h, e, "stream synchronisation");
     d->device_status = status;
     if (status != 0) return fail(h, LAZYEV_EDEVICE, "device status word = %d (1: wait timed out, 2: bad index)", status);
+    return LAZYEV_OK;
+}
+
+int lazyev_mri_histogram(lazyev_t* h, int unit_begin, int unit_count, long long* host_hist, int bins) {
+    if (!h || !host_hist) return LAZYEV_EINVAL;
+    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "mri_histogram before prefill");
+    if (unit_begin < 0 || unit_count <= 0 || unit_begin + unit_count > h->units)
+        return fail(h, LAZYEV_EINVAL, "unit range out of bounds");
+    if (bins < 2 || bins > kMaxHistBins) return fail(h, LAZYEV_EINVAL, "bins must be in [2, %d]", kMaxHistBins);
+    cudaError_t e = mri_histogram_launch(geometry(h), h->st, unit_begin, unit_count, h->n, bins, h->stage_hist, h->stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(host_hist, h->stage_hist, (size_t)bins * sizeof(long long), cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "MRI histogram");
+    h->launches += 1;
+    return LAZYEV_OK;
+}
+
+int lazyev_mri_quantile(lazyev_t* h, int unit_begin, int unit_count, double fraction, int* value, long long* recurring) {
+    if (!h || !value) return LAZYEV_EINVAL;
+    if (!(fraction > 0.0 && fraction <= 1.0)) return fail(h, LAZYEV_EINVAL, "fraction must be in (0, 1]");
+    std::vector<long long> hist(kMaxHistBins);
+    const int rc = lazyev_mri_histogram(h, unit_begin, unit_count, hist.data(), kMaxHistBins);
+    if (rc != LAZYEV_OK) return rc;
+    long long total = 0;
+    for (int b = 1; b < kMaxHistBins; ++b) total += hist[b];
+    if (recurring) *recurring = total;
+    *value = 0;
+    if (total == 0) return LAZYEV_OK;
+    // smallest v such that at least fraction * total of the re-activated tokens have MRI <= v
+    long long cum = 0;
+    for (int b = 1; b < kMaxHistBins; ++b) {
+        cum += hist[b];
+        if ((double)cum >= fraction * (double)total) {
+            *value = b;
+            break;
+        }
+    }
     return LAZYEV_OK;
 }
 

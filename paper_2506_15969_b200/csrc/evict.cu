@@ -16,13 +16,18 @@ namespace {
 //   H2 = 2 sigma(-1 / (MRI - 1))    (0 for MRI = 0 by definition and for MRI = 1 as the limit)
 //   Eq. (2): H1 + H2 when MRI != 0, H1 alone when MRI = 0.
 // 2 sigma(-x) is evaluated as 2 / (1 + exp(x)).
+// Modes: 0 = Eq. (2); 1 = H1 only; 2 = H2 only (the paper's ablations); 3 = Eq. (2) with
+// H2 = 2 sigma(-(MRI - 1)), a variant that decreases with MRI as the paper's prose asks.
 __device__ __forceinline__ double score_fn(int d, int mri, int mode) {
     double h1, h2 = 0.0;
     if (mri == 0) {
         h1 = d == 0 ? 1.0 : 0.0;
     } else {
         h1 = 2.0 / (1.0 + exp((double)d / (double)mri));
-        if (mri > 1) h2 = 2.0 / (1.0 + exp(1.0 / ((double)mri - 1.0)));
+        if (mode == 3)
+            h2 = 2.0 / (1.0 + exp((double)mri - 1.0));
+        else if (mri > 1)
+            h2 = 2.0 / (1.0 + exp(1.0 / ((double)mri - 1.0)));
     }
     if (mode == 1) return h1;
     if (mode == 2) return h2;
@@ -283,6 +288,42 @@ __global__ void score_kernel(Geometry geo, StateView st, int unit_begin, int uni
     }
 }
 
+// Histogram of MRI over the cached tokens of a range of units (Section 4, "Discussion about the
+// choice of W and alpha": W is read off the distribution of MRI).  hist[b] counts tokens with MRI = b
+// for b < bins - 1; the last bin takes every larger value.  Blocks stride over units, count the
+// first kHistSmemBins values in shared memory and flush what is non-zero with one atomic per bin.
+constexpr int kHistSmemBins = 8192;
+
+__global__ void __launch_bounds__(256) mri_histogram_kernel(Geometry geo, StateView st, int unit_begin,
+                                                           int unit_count, int n, int bins,
+                                                           unsigned long long* hist) {
+    __shared__ unsigned int local[kHistSmemBins];
+    const int nlocal = min(bins, kHistSmemBins);
+    for (int b = threadIdx.x; b < nlocal; b += blockDim.x) local[b] = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    for (int u = unit_begin + blockIdx.x; u < unit_begin + unit_count; u += gridDim.x) {
+        const int32_t* mri = st.mri + (size_t)u * geo.capacity;
+        for (int i0 = 0; i0 < n; i0 += blockDim.x) {
+            const int i = i0 + threadIdx.x;
+            const bool on = i < n;
+            const int v = on ? mri[i] : -1;
+            const int b = v < 0 ? 0 : min(v, bins - 1);
+            // most tokens share one value (0): one atomic per distinct value and warp
+            const unsigned peers = __match_any_sync(0xffffffffu, on ? b : -1);
+            if (on && (int)(__ffs(peers) - 1) == lane) {
+                if (b < nlocal)
+                    atomicAdd(&local[b], (unsigned)__popc(peers));
+                else
+                    atomicAdd(&hist[b], (unsigned long long)__popc(peers));
+            }
+        }
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < nlocal; b += blockDim.x)
+        if (local[b] != 0u) atomicAdd(&hist[b], (unsigned long long)local[b]);
+}
+
 }  // namespace
 
 size_t select_smem_bytes(int n_candidates) { return (size_t)n_candidates * sizeof(unsigned long long); }
@@ -308,6 +349,15 @@ cudaError_t score_launch(const Geometry& geo, StateView st, int unit_begin, int 
     const size_t total = (size_t)unit_count * geo.capacity;
     const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
     score_kernel<<<blocks, 256, 0, stream>>>(geo, st, unit_begin, unit_count, n, t, score_mode, out);
+    return cudaGetLastError();
+}
+
+cudaError_t mri_histogram_launch(const Geometry& geo, StateView st, int unit_begin, int unit_count, int n, int bins,
+                                 unsigned long long* hist, cudaStream_t stream) {
+    cudaError_t e = cudaMemsetAsync(hist, 0, (size_t)bins * sizeof(unsigned long long), stream);
+    if (e != cudaSuccess) return e;
+    const int blocks = unit_count < 148 * 4 ? unit_count : 148 * 4;
+    mri_histogram_kernel<<<blocks, 256, 0, stream>>>(geo, st, unit_begin, unit_count, n, bins, hist);
     return cudaGetLastError();
 }
 

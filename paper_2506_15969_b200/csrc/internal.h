@@ -64,4 +64,8 @@ cudaError_t compact_launch(const Geometry& geo, uint8_t* pool, StateView st, con
 cudaError_t score_launch(const Geometry& geo, StateView st, int unit_begin, int unit_count, int n, int t,
                          int score_mode, double* out, cudaStream_t stream);
 
+// hist[b] (b < bins - 1) = cached tokens of the unit range with MRI = b; hist[bins - 1] = the rest.
+cudaError_t mri_histogram_launch(const Geometry& geo, StateView st, int unit_begin, int unit_count, int n, int bins,
+                                 unsigned long long* hist, cudaStream_t stream);
+
 }  // namespace lzk

@@ -62,7 +62,8 @@ def test_host_side_configuration_and_sizes():
     assert lib.lazyev_set_budget(h, 4096) == binding.OK
     assert lib.lazyev_set_budget(h, 8193) == binding.EINVAL
     assert lib.lazyev_set_budget(h, 132) == binding.EINVAL
-    assert lib.lazyev_set_score_mode(h, 3) == binding.EINVAL
+    assert lib.lazyev_set_score_mode(h, 3) == binding.OK
+    assert lib.lazyev_set_score_mode(h, 4) == binding.EINVAL
     assert lib.lazyev_set_splits(h, 9) == binding.EINVAL and lib.lazyev_set_splits(h, 3) == binding.OK
     kv, st, sc = C.c_size_t(), C.c_size_t(), C.c_size_t()
     assert lib.lazyev_query_sizes(h, C.byref(kv), C.byref(st), C.byref(sc)) == binding.OK

@@ -120,7 +120,8 @@ def test_lockstep_with_evictions(splits):
 
 def test_protected_tokens_and_score_variants():
     cfg = traces.tiny_config(n_recent=8, n_initial=4, budget=130, window=16, prefill=100)
-    for mode in (binding.SCORE_H1_PLUS_H2, binding.SCORE_H1_ONLY, binding.SCORE_H2_ONLY):
+    for mode in (binding.SCORE_H1_PLUS_H2, binding.SCORE_H1_ONLY, binding.SCORE_H2_ONLY,
+                 binding.SCORE_H1_PLUS_H2_DECREASING):
         ls = lockstep(cfg, seed=4, sample_units=[0, 3, 7], score_mode=mode)
         rep = ls.run(160)
         ls.assert_ok(jaccard=0.99)
@@ -190,6 +191,27 @@ def test_config1_full_trace():
         kept = set(ls.shadow[i].pos.tolist())
         alive = sum(1 for p in np.nonzero(planted[i])[0] if int(p) in kept)
         assert alive >= 30, alive
+
+
+def test_mri_histogram_and_quantile_match_the_oracle():
+    """The live distribution of MRI (the paper's offline rule for choosing W): bit-exact counts."""
+    from oracle import lazyev_oracle as orc
+    cfg = traces.tiny_config(budget=400, window=32, prefill=200, alpha=0.004)
+    ls = lockstep(cfg, seed=9, sample_units=range(cfg.units), pure=False)
+    ls.run(230)
+    ls.assert_ok()
+    mri = [sh.MRI for sh in ls.shadow]
+    assert sum(int((m > 0).sum()) for m in mri) > 200              # plenty of re-activated tokens
+    for bins in (2, 17, 64, 9000, 65536):
+        assert np.array_equal(ls.eng.mri_histogram(bins), orc.mri_histogram(mri, bins)), bins
+    assert np.array_equal(ls.eng.mri_histogram(64, 3, 2), orc.mri_histogram(mri[3:5], 64))
+    for frac in (0.1, 0.5, 0.8, 1.0):
+        assert ls.eng.mri_quantile(frac) == orc.mri_quantile(mri, frac)
+        assert ls.eng.mri_quantile(frac, 5, 1) == orc.mri_quantile(mri[5:6], frac)
+    with pytest.raises(binding.LazyEvError):
+        ls.eng.mri_histogram(1)
+    with pytest.raises(binding.LazyEvError):
+        ls.eng.mri_histogram(16, 7, 2)
 
 
 def test_call_order_errors_and_capacity():

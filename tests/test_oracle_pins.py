@@ -233,6 +233,51 @@ def test_score_against_tanh_identity_and_properties():
         assert vec[i] == float(orc.importance(t, ts[i], mri[i]))
 
 
+def test_decreasing_h2_variant_has_the_properties_the_appendix_requires():
+    """The appendix on the score's formulation asks for a monotonically decreasing function
+    with values in [0, 1], and Section 4 for "smaller MRI, higher score": the variant
+    2*sigma(-(MRI - 1)) has them, the printed H2 does not (it increases with MRI)."""
+    e = math.e
+    assert float(orc.h2_decreasing(0)) == 0.0                       # never re-activated: stays 0 as in the text
+    assert float(orc.h2_decreasing(1)) == 1.0                       # 2*sigma(0)
+    assert float(orc.h2_decreasing(2)) == pytest.approx(2.0 / (1.0 + e), abs=1e-15)
+    assert float(orc.h2_decreasing(4)) == pytest.approx(1.0 - math.tanh(1.5), abs=1e-15)
+    grid = np.arange(1, 60)
+    dec, printed = orc.h2_decreasing(grid), orc.h2_score(grid)
+    assert (np.diff(dec) < 0).all() and (dec >= 0).all() and (dec <= 1).all()
+    assert (np.diff(printed) > 0).all()                             # the printed formula goes the other way
+    assert float(orc.h2_decreasing(10 ** 6)) == 0.0
+    # inside Eq. (2): H1 + variant when MRI != 0, H1 alone when MRI = 0
+    I = lambda d, mri: float(orc.importance(100, 100 - d, mri, "h1+h2dec"))
+    assert I(2, 2) == pytest.approx(2.0 / (1.0 + e) + 2.0 / (1.0 + e), abs=1e-15)
+    assert I(0, 0) == 1.0 and I(7, 0) == 0.0
+    # two tokens, equally overdue relative to their intervals: the frequent one now ranks higher
+    assert I(3, 3) > I(30, 30) and float(orc.importance(100, 97, 3)) < float(orc.importance(100, 70, 30))
+
+
+def test_mri_histogram_and_quantile_closed_forms_and_library_routine():
+    """One token per MRI value 1..100 (plus never re-activated ones): the 80 % value is 80;
+    on random data the rule equals numpy's inverted-CDF percentile of the re-activated tokens."""
+    a = [np.arange(0, 51), np.concatenate([np.arange(51, 101), np.zeros(500, dtype=np.int64)])]
+    assert orc.mri_quantile(a, 0.8) == (80, 100)
+    assert orc.mri_quantile(a, 1.0) == (100, 100) and orc.mri_quantile(a, 0.005) == (1, 100)
+    assert orc.mri_quantile([np.zeros(7)], 0.8) == (0, 0)
+    h = orc.mri_histogram(a, 64)
+    assert h[0] == 501 and (h[1:63] == 1).all() and h[63] == 100 - 62 and h.sum() == 601
+    rng = np.random.default_rng(3)
+    for _ in range(20):
+        arrs = [rng.integers(0, 300, size=rng.integers(1, 400)) * (rng.random(1) < 0.9) for _ in range(3)]
+        pooled = np.concatenate(arrs)
+        pooled = pooled[pooled >= 1]
+        frac = float(rng.uniform(0.05, 1.0))
+        if pooled.size:
+            want = int(np.percentile(pooled, 100 * frac, method="inverted_cdf"))
+            assert orc.mri_quantile(arrs, frac) == (want, pooled.size)
+        hist = orc.mri_histogram(arrs, 128)
+        assert hist.sum() == sum(len(x) for x in arrs)
+        assert np.array_equal(hist[:127], np.bincount(np.concatenate(arrs), minlength=300)[:127])
+
+
 def test_elapsed_beyond_mri_is_evicted_first():
     """Two tokens with the same MRI = 10: the one last seen 50 steps ago goes
     before the one last seen 5 steps ago (Introduction: evict when the elapsed
