@@ -193,6 +193,30 @@ def test_config1_full_trace():
         assert alive >= 30, alive
 
 
+@pytest.mark.parametrize("prefill,splits", [(8150, 1), (9000, 1), (16900, 2), (16900, 0)])
+def test_full_cache_long_contexts(prefill, splits):
+    """No eviction (budget above prompt + steps, the FullKV setting) at lengths where a unit's logits
+    fill tensor memory and spill to shared memory (8193..9040 tokens, one block per unit) and where
+    a unit needs a cluster (16.9 k tokens)."""
+    cfg = traces.tiny_config(batch=1, layers=2, q_heads=14, kv_heads=2, budget=prefill + 200, window=64,
+                             prefill=prefill, n_recent=64)
+    ls = lockstep(cfg, seed=15, sample_units=[0, 3], pure=False, splits=splits)
+    ls.run(48, check_every=1)
+    ls.assert_ok()
+    inf = ls.eng.info()
+    assert ls.rep.evictions == 0 and inf.n == prefill + 48
+    assert splits == 0 or inf.splits == splits
+
+
+def test_per_step_eviction_window_of_one():
+    """W = 1: an eviction decision at every step (the greedy setting the paper contrasts with)."""
+    cfg = traces.tiny_config(budget=120, window=1, n_recent=1, prefill=100)
+    ls = lockstep(cfg, seed=16, sample_units=[0, 2, 7])
+    ls.run(90)
+    ls.assert_ok(jaccard=0.99)
+    assert ls.rep.evictions == 90 - 20 and ls.eng.info().n == 120
+
+
 def test_mri_histogram_and_quantile_match_the_oracle():
     """The live distribution of MRI (the paper's offline rule for choosing W): bit-exact counts."""
     from oracle import lazyev_oracle as orc
