@@ -225,6 +225,20 @@ typedef struct lazyev_dump {
 int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* dump);
 
 /*
+ * Resume from a snapshot taken with lazyev_dump_state (checkpoint / restore; the paper has
+ * no counterpart, its method keeps no state beyond TS and MRI of Eq. (1) and the cache).
+ * Valid on a bound handle instead of lazyev_prefill().  `snap` must cover all units
+ * (unit_begin = 0, unit_count = units) with pos, ts, mri, k and v set (host arrays laid out
+ * as dump_state writes them, row stride snap->capacity; pbar optional, score ignored) and
+ * its n and t; `prefill` is the prompt length of the original run (positions of new tokens
+ * continue from prefill + t).  The handle may have another capacity than the one the
+ * snapshot came from as long as n fits.  Decoding then continues exactly as the original
+ * handle would have.  Synchronises the stream; a slow path (one host-to-device copy per page).
+ * Errors: EINVAL (partial snapshot, sizes), ESTATE (not bound, or already holds a cache), ECUDA.
+ */
+int lazyev_load_state(lazyev_t* h, const lazyev_dump_t* snap, int prefill);
+
+/*
  * Distribution of the recurrence intervals in the live cache (Section 4, "Discussion about
  * the choice of W and alpha": the paper sets W to the MRI value below which 80 % of the
  * tokens fall, found offline).  host_hist[b], b < bins - 1, receives the number of cached

@@ -61,6 +61,7 @@ _PROTOS = {
     "lazyev_evict_static": [C.c_void_p, C.POINTER(C.c_int)],
     "lazyev_get_info": [C.c_void_p, C.POINTER(Info)],
     "lazyev_dump_state": [C.c_void_p, C.POINTER(Dump)],
+    "lazyev_load_state": [C.c_void_p, C.POINTER(Dump), C.c_int],
     "lazyev_mri_histogram": [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int],
     "lazyev_mri_quantile": [C.c_void_p, C.c_int, C.c_int, C.c_double, C.POINTER(C.c_int), C.POINTER(C.c_longlong)],
     "lazyev_set_profiling": [C.c_void_p, C.c_int],
@@ -190,6 +191,18 @@ class Engine:
         n = C.c_int()
         self._check(lib().lazyev_evict_static(self._h, C.byref(n)))
         return n.value
+
+    def load_state(self, snap: dict, prefill: int) -> None:
+        """lazyev_load_state from a dict as returned by dump_state(kv=True) over all units."""
+        cnt, n = snap["pos"].shape
+        d = Dump(unit_begin=0, unit_count=cnt, t=snap["t"], n=n, capacity=n)
+        keep = {}
+        for name, dt in (("pos", np.int32), ("ts", np.int32), ("mri", np.int32), ("pbar", np.float32),
+                         ("k", np.uint16), ("v", np.uint16)):
+            if name in snap:
+                keep[name] = np.ascontiguousarray(snap[name], dtype=dt)
+                setattr(d, name, keep[name].ctypes.data)
+        self._check(lib().lazyev_load_state(self._h, C.byref(d), prefill))
 
     def mri_histogram(self, bins: int, unit_begin: int = 0, unit_count: Optional[int] = None):
         """lazyev_mri_histogram: int64 counts per MRI value (last bin: everything larger)."""

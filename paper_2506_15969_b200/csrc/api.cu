@@ -723,6 +723,51 @@ int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* d) {
     return LAZYEV_OK;
 }
 
+int lazyev_load_state(lazyev_t* h, const lazyev_dump_t* d, int prefill) {
+    if (!h || !d) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "load_state before bind");
+    if (h->prefilled) return fail(h, LAZYEV_ESTATE, "load_state on a handle that already holds a cache");
+    if (d->unit_begin != 0 || d->unit_count != h->units) return fail(h, LAZYEV_EINVAL, "the snapshot must cover all %d units", h->units);
+    if (!d->pos || !d->ts || !d->mri || !d->k || !d->v) return fail(h, LAZYEV_EINVAL, "pos, ts, mri, k and v are required");
+    if (d->n <= 0 || d->n > h->capacity || d->capacity < d->n || d->t < 0 || prefill <= 0)
+        return fail(h, LAZYEV_EINVAL, "snapshot sizes out of range (n = %d, capacity here = %d)", d->n, h->capacity);
+    const size_t scap = (size_t)d->capacity, width = (size_t)d->n * 4;
+    cudaError_t e = cudaMemcpy2DAsync(h->st.pos, (size_t)h->capacity * 4, d->pos, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(h->st.ts, (size_t)h->capacity * 4, d->ts, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaMemcpy2DAsync(h->st.mri, (size_t)h->capacity * 4, d->mri, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess && d->pbar) e = cudaMemcpy2DAsync(h->st.pbar, (size_t)h->capacity * 4, d->pbar, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "state upload");
+    // K / V rows: swizzled into pages on the host, one page per copy
+    const int np = (d->n + kPageTokens - 1) / kPageTokens;
+    std::vector<int32_t> table((size_t)h->units * h->pages_per_unit);
+    e = cudaMemcpyAsync(table.data(), h->st.page_table, table.size() * 4, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "page table download");
+    std::vector<uint8_t> page(kPageBytes);
+    for (int u = 0; u < h->units; ++u) {
+        for (int pg = 0; pg < np; ++pg) {
+            memset(page.data(), 0, kPageBytes);
+            for (int r = 0; r < kPageTokens && pg * kPageTokens + r < d->n; ++r) {
+                const size_t slot = (size_t)u * scap + (size_t)pg * kPageTokens + r;
+                for (int c = 0; c < kChunksPerRow; ++c) {
+                    uint8_t* kd = page.data() + r * kRowBytes + swz_chunk(c, r) * 16;
+                    memcpy(kd, (const uint8_t*)d->k + slot * kRowBytes + c * 16, 16);
+                    memcpy(kd + kPageHalfBytes, (const uint8_t*)d->v + slot * kRowBytes + c * 16, 16);
+                }
+            }
+            const int32_t pp = table[(size_t)u * h->pages_per_unit + pg];
+            e = cudaMemcpyAsync(h->pool + (size_t)pp * kPageBytes, page.data(), kPageBytes, cudaMemcpyHostToDevice, h->stream);
+            if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);      // the staging page is reused
+            if (e != cudaSuccess) return cuda_fail(h, e, "page upload");
+        }
+    }
+    h->prefilled = true;
+    h->prefill = prefill;
+    h->n = d->n;
+    h->t = d->t;
+    return LAZYEV_OK;
+}
+
 int lazyev_mri_histogram(lazyev_t* h, int unit_begin, int unit_count, long long* host_hist, int bins) {
     if (!h || !host_hist) return LAZYEV_EINVAL;
     if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "mri_histogram before prefill");

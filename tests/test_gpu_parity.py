@@ -238,6 +238,46 @@ def test_mri_histogram_and_quantile_match_the_oracle():
         ls.eng.mri_histogram(16, 7, 2)
 
 
+def test_resume_from_a_snapshot_continues_bit_for_bit():
+    """dump_state -> load_state into a fresh handle (with a larger capacity): the resumed run must
+    produce the same outputs, statistics, evictions and cache as the run that was never stopped."""
+    from tests.harness import make_engine
+    cfg = traces.tiny_config()
+    gen = traces.TraceGen(cfg, 21, device="cuda")
+    a = make_engine(cfg)
+    k, v = gen.prefill()
+    shape = (cfg.layers, cfg.batch, cfg.kv_heads, cfg.prefill, 128)
+    a.prefill(k.view(shape), v.view(shape))
+    out_a = torch.empty(cfg.layers, cfg.batch, cfg.q_heads, 128, dtype=torch.bfloat16, device="cuda")
+    out_b = torch.empty_like(out_a)
+    for _ in range(5):                                       # 160 steps: three evictions, t not on a window edge + 0
+        q, kn, vn = gen.steps(32)
+        for s in range(32):
+            a.decode_step(q[s], kn[s], vn[s], out_a)
+    q, kn, vn = gen.steps(13)
+    for s in range(13):
+        a.decode_step(q[s], kn[s], vn[s], out_a)
+    snap = a.dump_state(kv=True)
+    big = dataclasses.replace(cfg, prefill=cfg.prefill + 200)          # another capacity than the original
+    b = make_engine(big)
+    with pytest.raises(binding.LazyEvError):
+        b.load_state({k2: (v2[:3] if hasattr(v2, "shape") else v2) for k2, v2 in snap.items()}, cfg.prefill)   # partial
+    b.load_state(snap, cfg.prefill)
+    assert (b.info().t, b.info().n) == (173, snap["n"])
+    with pytest.raises(binding.LazyEvError):
+        b.load_state(snap, cfg.prefill)                                  # already holds a cache
+    for _ in range(3):
+        q, kn, vn = gen.steps(32)
+        for s in range(32):
+            a.decode_step(q[s], kn[s], vn[s], out_a)
+            b.decode_step(q[s], kn[s], vn[s], out_b)
+            assert torch.equal(out_a, out_b)
+    da, db = a.dump_state(kv=True), b.dump_state(kv=True)
+    assert a.info().evictions == b.info().evictions + 3 and da["n"] == db["n"]
+    for key in ("pos", "ts", "mri", "pbar", "k", "v"):
+        assert np.array_equal(da[key], db[key]), key
+
+
 def test_call_order_errors_and_capacity():
     cfg = traces.tiny_config(batch=1, layers=1)
     eng = binding.Engine(1, 8, 2, 128, 160, 32, 0.01, max_prefill=96)
