@@ -137,8 +137,10 @@ int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens);
  */
 int lazyev_decode_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out);
 
-/* The same step with HOST buffers (pinned memory recommended): copies the three
- * inputs to the device, runs the step, copies `out` back and synchronises the stream. */
+/* The same step with HOST buffers (pinned memory recommended; pageable memory works but
+ * serialises the copies): copies the inputs to the device, runs the step, copies `out` back and
+ * synchronises.  Queries and outputs move in unit ranges on two internal copy streams
+ * (created at the first call) while the decode launches of the other ranges run. */
 int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out);
 
 /*

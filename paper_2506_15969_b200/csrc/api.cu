@@ -14,6 +14,8 @@
 
 using namespace lzk;
 
+constexpr int kHostChunks = 4;            // unit ranges the host-buffer entry point pipelines copies over
+
 struct lazyev {
     // configuration
     int layers = 0, batch = 1, q_heads = 0, kv_heads = 0, head_dim = 0;
@@ -35,6 +37,9 @@ struct lazyev {
     uint8_t* stage_out = nullptr;
     double* stage_score = nullptr;
     unsigned long long* stage_hist = nullptr;
+    // host-buffer entry point: copy streams and events, created at its first call
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_in[kHostChunks + 1] = {}, ev_done[kHostChunks + 1] = {}, ev_ready = nullptr;
     // progress
     int t = 0, n = 0, prefill = 0;
     long long launches = 0, evictions = 0;
@@ -239,7 +244,14 @@ int run_evict(lazyev_t* h, int* evicted) {
     return LAZYEV_OK;
 }
 
-int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out) {
+// Host side of a pipelined step: queries come from and outputs go to host memory in unit ranges, on
+// two copy streams, while the decode launches of the other ranges run.
+struct HostPipe {
+    const uint8_t* q_host;
+    uint8_t* out_host;
+};
+
+int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out, const HostPipe* pipe = nullptr) {
     if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
     if (h->n + 1 > h->capacity) return fail(h, LAZYEV_ECAPACITY, "cache full (%d slots per unit)", h->capacity);
     const Geometry geo = geometry(h);
@@ -324,16 +336,49 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
         // algorithmic bytes: every cached K and V row read once, one probability written per token,
         // the queries read and the outputs written
         SpanGuard g(h, kSpanDecode, (double)h->units * ((double)n * (2 * kRowBytes + 4) + 2.0 * h->group * kRowBytes));
-        DecodeArgs a{h->pool, h->st, q, out, n, t, 0, main_units};
-        e = decode_launch(c, plan, clusters, a, h->stream);
-        if (e == cudaSuccess && shape.tail_units > 0) {
-            DecodeArgs b{h->pool, h->st, q, out, n, t, main_units, shape.tail_units};
-            e = decode_launch(c, tail_plan, shape.tail_units, b, h->stream);
+        // Unit ranges: the main launch as one range, or (host buffers) as up to kHostChunks ranges of whole
+        // rounds so that copies of one range overlap the kernel of another; then the last round's units.
+        int begin[kHostChunks + 1], count[kHostChunks + 1], ranges = 0;
+        const int rounds = (main_units + clusters - 1) / clusters;
+        const int parts = pipe ? (rounds < kHostChunks ? rounds : kHostChunks) : 1;
+        for (int r = 0; r < parts; ++r) {
+            const int b = (int)((long long)rounds * r / parts) * clusters;
+            int e2 = (int)((long long)rounds * (r + 1) / parts) * clusters;
+            if (e2 > main_units) e2 = main_units;
+            begin[ranges] = b;
+            count[ranges++] = e2 - b;
+        }
+        if (shape.tail_units > 0) {
+            begin[ranges] = main_units;
+            count[ranges++] = shape.tail_units;
+        }
+        const size_t unit_bytes = (size_t)h->group * kRowBytes;
+        if (pipe) {
+            for (int r = 0; r < ranges && e == cudaSuccess; ++r) {
+                e = cudaMemcpyAsync((uint8_t*)const_cast<void*>(q) + begin[r] * unit_bytes, pipe->q_host + begin[r] * unit_bytes,
+                                    count[r] * unit_bytes, cudaMemcpyHostToDevice, h->copy_in);
+                if (e == cudaSuccess) e = cudaEventRecord(h->ev_in[r], h->copy_in);
+            }
+        }
+        for (int r = 0; r < ranges && e == cudaSuccess; ++r) {
+            const bool is_tail = shape.tail_units > 0 && r == ranges - 1;
+            if (pipe) e = cudaStreamWaitEvent(h->stream, h->ev_in[r], 0);
+            if (e != cudaSuccess) break;
+            DecodeArgs a{h->pool, h->st, q, out, n, t, begin[r], count[r]};
+            e = decode_launch(c, is_tail ? tail_plan : plan, is_tail ? count[r] : (clusters < count[r] ? clusters : count[r]), a,
+                              h->stream);
             h->launches += 1;
+            if (pipe && e == cudaSuccess) {
+                e = cudaEventRecord(h->ev_done[r], h->stream);
+                if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_done[r], 0);
+                if (e == cudaSuccess)
+                    e = cudaMemcpyAsync(pipe->out_host + begin[r] * unit_bytes, (uint8_t*)out + begin[r] * unit_bytes,
+                                        count[r] * unit_bytes, cudaMemcpyDeviceToHost, h->copy_out);
+            }
         }
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "decode kernel launch");
-    h->launches += 2;
+    h->launches += 1;      // the append kernel
     h->last_plan = plan;
     h->last_tail_units = shape.tail_units;
     h->last_tail_splits = shape.tail_splits;
@@ -555,17 +600,34 @@ int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const
     if (!h) return LAZYEV_EINVAL;
     if (!q || !k_new || !v_new || !out) return fail(h, LAZYEV_EINVAL, "null pointer");
     if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
-    const size_t qbytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
+    cudaError_t e = cudaSuccess;
+    if (!h->copy_in) {      // first call: the two copy streams and their events
+        e = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking);
+        for (int i = 0; i <= kHostChunks && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming);
+        }
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_ready, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail(h, e, "creating the copy streams");
+    }
+    // The copy streams start after everything queued on the bound stream so far (an earlier step's
+    // kernels may still read the staging buffers).
+    e = cudaEventRecord(h->ev_ready, h->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_in, h->ev_ready, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_ready, 0);
     const size_t kbytes = (size_t)h->layers * h->batch * h->kv_heads * kRowBytes;
-    cudaError_t e = cudaMemcpyAsync(h->stage_q, q, qbytes, cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_k, k_new, kbytes, cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_v, v_new, kbytes, cudaMemcpyHostToDevice, h->stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "host-to-device copy");
-    const int rc = run_step(h, h->stage_q, h->stage_k, h->stage_v, h->stage_out);
+    const HostPipe pipe{(const uint8_t*)q, (uint8_t*)out};
+    const int rc = run_step(h, h->stage_q, h->stage_k, h->stage_v, h->stage_out, &pipe);
+    // both streams are drained even after an error, so that no copy is left in flight on the caller's buffers
+    cudaError_t e1 = cudaStreamSynchronize(h->copy_in), e2 = cudaStreamSynchronize(h->copy_out);
+    e = cudaStreamSynchronize(h->stream);
     if (rc != LAZYEV_OK) return rc;
-    e = cudaMemcpyAsync(out, h->stage_out, qbytes, cudaMemcpyDeviceToHost, h->stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
-    if (e != cudaSuccess) return cuda_fail(h, e, "device-to-host copy");
+    if (e1 != cudaSuccess || e2 != cudaSuccess || e != cudaSuccess)
+        return cuda_fail(h, e1 != cudaSuccess ? e1 : (e2 != cudaSuccess ? e2 : e), "copies of the host-buffer step");
     return LAZYEV_OK;
 }
 
@@ -836,6 +898,13 @@ int lazyev_destroy(lazyev_t* h) {
         cudaEventDestroy(sp.stop);
     }
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
+    if (h->copy_in) cudaStreamDestroy(h->copy_in);
+    if (h->copy_out) cudaStreamDestroy(h->copy_out);
+    for (int i = 0; i <= kHostChunks; ++i) {
+        if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+        if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
+    }
+    if (h->ev_ready) cudaEventDestroy(h->ev_ready);
     delete h;
     return LAZYEV_OK;
 }
