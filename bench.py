@@ -105,6 +105,17 @@ def first_eviction_step(cfg) -> int:
     return t
 
 
+def steady_state_start(cfg, timed_steps: int) -> int:
+    """Decode steps replayed untimed: up to the first eviction for a fixed budget (the cache then
+    cycles between B and B + W); for a budget that grows with the length, up to the end of the trace
+    minus the timed steps, where the cache is largest."""
+    first = first_eviction_step(cfg)
+    if not cfg.budget_frac_tenths:
+        return first
+    late = (cfg.steps - timed_steps - cfg.window) // cfg.window * cfg.window
+    return max(first, late)
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -282,7 +293,7 @@ def run_ours(args):
             count -= c
         return ms
 
-    start = first_eviction_step(cfg) if args.start_step < 0 else args.start_step
+    start = steady_state_start(cfg, args.steps) if args.start_step < 0 else args.start_step
     untimed = max(start, args.warmup, 3)
     run_steps(untimed)                                   # replay + warm-up, not timed
     eng.synchronize()

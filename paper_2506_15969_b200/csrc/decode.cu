@@ -58,7 +58,7 @@ struct DecodeParams {
     int n, t;
     float alpha, scale_log2, inv_group;
     int splits, stages, pages_per_cta, logit_stride, tmem_pages, tmem_cols;
-    int off_logits, off_xchg, off_wml, off_misc, off_bars;
+    int off_logits, off_xchg, off_wml, off_slots, off_misc, off_bars;
 };
 
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s is a failure, not a delay
@@ -104,10 +104,12 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
     float* spill = reinterpret_cast<float*>(smem + p.off_logits);       // logits of the pages beyond tensor memory
     Xchg* xchg = reinterpret_cast<Xchg*>(smem + p.off_xchg);          // [2], alternating per unit
     float* wml = reinterpret_cast<float*>(smem + p.off_wml);            // [NW][16]: m[8], l[8] per warp
+    float* slots = reinterpret_cast<float*>(smem + p.off_slots);        // [NW][8][kXchgRow]: O^T of every warp
     float* lse_s = reinterpret_cast<float*>(smem + p.off_misc);         // [8]
     float* sc_s = lse_s + kMaxGroup;                                    // [splits <= 8][8]
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sc_s + 8 * kMaxGroup);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sc_s + 8 * kMaxGroup) + 1;
+    float* scw = sc_s + 8 * kMaxGroup;                                  // [NW <= 8][8]: scale of every warp's partial sums
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(scw + 8 * kMaxGroup);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(scw + 8 * kMaxGroup) + 1;
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + p.off_bars);
     uint64_t* empty = full + p.stages;
 
@@ -296,17 +298,22 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
             }
         };
 
-        for (int u = p.unit_begin + cluster_id; u < p.unit_end; u += n_clusters, ++it) {
-            // Q^T as the B operand: b0 = Q[head g][16 ks + 2 qd, +1], b1 = the same 8 dims further
-            uint32_t qb[8][2];
-            {
-                const __nv_bfloat16* qrow = p.q + ((size_t)u * G + g) * kHeadDim;
+        // Q^T as the B operand: b0 = Q[head g][16 ks + 2 qd, +1], b1 = the same 8 dims further.  The
+        // fragments of the next unit are fetched while the current one streams.
+        uint32_t qb[8][2];
+        auto load_q = [&](int u, uint32_t (&dst)[8][2]) {
+            const __nv_bfloat16* qrow = p.q + ((size_t)u * G + g) * kHeadDim;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    qb[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * qd) : 0u;
-                    qb[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * qd) : 0u;
-                }
+            for (int ks = 0; ks < 8; ++ks) {
+                dst[ks][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * qd) : 0u;
+                dst[ks][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * qd) : 0u;
             }
+        };
+        if (my_units > 0) load_q(p.unit_begin + cluster_id, qb);
+
+        for (int u = p.unit_begin + cluster_id; u < p.unit_end; u += n_clusters, ++it) {
+            uint32_t qn[8][2] = {};
+            if (u + n_clusters < p.unit_end) load_q(u + n_clusters, qn);
             float mref0 = -INFINITY, mref1 = -INFINITY, l0 = 0.f, l1 = 0.f;
             float o[8][4];      // O^T: [m-tile][(dim g, h0), (dim g, h1), (dim g + 8, h0), (dim g + 8, h1)]
 #pragma unroll
@@ -410,6 +417,10 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
             st_base = (st_base + (uint32_t)npg) % NS;
 
             // ---- merge the warps of this block ---------------------------------
+            // Every warp leaves its (reference, l) pair and its unscaled O^T in a slot of its own; after
+            // one barrier 8 x NW threads turn the references into per-warp scales and the block's
+            // (reference, l), and after a second one all threads add the slots up in warp order (the
+            // sum is the same in every run).
 #pragma unroll
             for (int s = 4; s < 32; s <<= 1) {
                 l0 += __shfl_xor_sync(0xffffffffu, l0, s);
@@ -421,48 +432,45 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 wml[warp * 16 + 8 + h0] = l0;
                 wml[warp * 16 + 8 + h1] = l1;
             }
-            named_barrier_sync(1, kConsumers);
-            float mc0 = -INFINITY, mc1 = -INFINITY, lc0 = 0.f, lc1 = 0.f;
+            {
+                float* slot = slots + warp * (kMaxGroup * kXchgRow);
 #pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                mc0 = fmaxf(mc0, wml[w * 16 + h0]);
-                mc1 = fmaxf(mc1, wml[w * 16 + h1]);
-            }
-#pragma unroll
-            for (int w = 0; w < NW; ++w) {
-                const float m0 = wml[w * 16 + h0], m1 = wml[w * 16 + h1];
-                lc0 += m0 == -INFINITY ? 0.f : wml[w * 16 + 8 + h0] * fast_exp2(m0 - mc0);
-                lc1 += m1 == -INFINITY ? 0.f : wml[w * 16 + 8 + h1] * fast_exp2(m1 - mc1);
-            }
-            const float f0 = mref0 == -INFINITY ? 0.f : fast_exp2(mref0 - mc0);
-            const float f1 = mref1 == -INFINITY ? 0.f : fast_exp2(mref1 - mc1);
-            Xchg* xb = xchg + (it & 1);
-            for (int w = 0; w < NW; ++w) {     // fixed order: the sum is the same in every run
-                if (warp == w) {
-#pragma unroll
-                    for (int mt = 0; mt < 8; ++mt) {
-                        float* d0 = &xb->o[h0][16 * mt + g];
-                        float* d1 = &xb->o[h1][16 * mt + g];
-                        if (w == 0) {
-                            d0[0] = o[mt][0] * f0;
-                            d1[0] = o[mt][1] * f1;
-                            d0[8] = o[mt][2] * f0;
-                            d1[8] = o[mt][3] * f1;
-                        } else {
-                            d0[0] += o[mt][0] * f0;
-                            d1[0] += o[mt][1] * f1;
-                            d0[8] += o[mt][2] * f0;
-                            d1[8] += o[mt][3] * f1;
-                        }
-                    }
+                for (int mt = 0; mt < 8; ++mt) {
+                    float* d0 = slot + h0 * kXchgRow + 16 * mt + g;
+                    float* d1 = slot + h1 * kXchgRow + 16 * mt + g;
+                    d0[0] = o[mt][0];
+                    d1[0] = o[mt][1];
+                    d0[8] = o[mt][2];
+                    d1[8] = o[mt][3];
                 }
-                named_barrier_sync(1, kConsumers);
             }
-            if (warp == 0 && g == 0) {
-                xb->m[h0] = mc0;
-                xb->m[h1] = mc1;
-                xb->l[h0] = lc0;
-                xb->l[h1] = lc1;
+            named_barrier_sync(1, kConsumers);
+            Xchg* xb = xchg + (it & 1);
+            if (ctid < kMaxGroup * NW) {
+                const int w = ctid >> 3, h = ctid & 7;
+                float mc = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < NW; ++k) mc = fmaxf(mc, wml[k * 16 + h]);
+                const float mw = wml[w * 16 + h];
+                scw[w * kMaxGroup + h] = mw == -INFINITY ? 0.f : fast_exp2(mw - mc);
+                if (w == 0) {
+                    float lc = 0.f;
+#pragma unroll
+                    for (int k = 0; k < NW; ++k) {
+                        const float mk = wml[k * 16 + h];
+                        lc += mk == -INFINITY ? 0.f : wml[k * 16 + 8 + h] * fast_exp2(mk - mc);
+                    }
+                    xb->m[h] = mc;
+                    xb->l[h] = lc;
+                }
+            }
+            named_barrier_sync(1, kConsumers);
+            for (int e = ctid; e < kMaxGroup * kHeadDim; e += kConsumers) {
+                const int h = e >> 7, d = e & (kHeadDim - 1);
+                float acc = 0.f;
+#pragma unroll
+                for (int k = 0; k < NW; ++k) acc += slots[k * (kMaxGroup * kXchgRow) + h * kXchgRow + d] * scw[k * kMaxGroup + h];
+                xb->o[h][d] = acc;
             }
             if (clustered) {
                 cluster_arrive();
@@ -501,6 +509,11 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                         acc += ld_rank_f32(&xb->o[gg][d], r, clustered) * sc_s[r * kMaxGroup + gg];
                     p.out[((size_t)u * G + gg) * kHeadDim + d] = __float2bfloat16_rn(acc);
                 }
+            }
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                qb[ks][0] = qn[ks][0];
+                qb[ks][1] = qn[ks][1];
             }
             // No barrier here: lse_s and sc_s are rewritten only after the barriers of the next unit's
             // merge, the exchange buffer alternates, and every logit slot is read and rewritten by
@@ -573,13 +586,15 @@ static size_t layout(const DecodeConfig& c, int np, int s, int ns, DecodePlan* p
     off += 2 * sizeof(Xchg);
     plan->off_wml = (int)off;
     off += 4 * kMaxGroups * 16 * sizeof(float);
+    plan->groups = c.force_groups > 0 ? c.force_groups : 2;
+    plan->off_slots = (int)off;
+    off += (size_t)4 * plan->groups * kMaxGroup * kXchgRow * sizeof(float);
     plan->off_misc = (int)off;
-    off += 128 * sizeof(float);
+    off += 256 * sizeof(float);
     plan->off_bars = (int)off;
     off += 2 * (size_t)ns * sizeof(uint64_t);
     plan->splits = s;
     plan->stages = ns;
-    plan->groups = c.force_groups > 0 ? c.force_groups : 2;
     plan->pages_per_cta = ppc;
     plan->logit_stride = ls;
     plan->tmem_pages = tp;
@@ -645,6 +660,7 @@ cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clu
     p.off_logits = plan.off_logits;
     p.off_xchg = plan.off_xchg;
     p.off_wml = plan.off_wml;
+    p.off_slots = plan.off_slots;
     p.off_misc = plan.off_misc;
     p.off_bars = plan.off_bars;
     return plan.groups == 2 ? launch_impl<2>(p, plan, clusters, stream, nullptr)

@@ -16,7 +16,7 @@ struct DecodeConfig {
 
 struct DecodePlan {
     int splits, stages, groups, pages_per_cta, logit_stride, tmem_pages, tmem_cols;
-    int off_logits, off_xchg, off_wml, off_misc, off_bars, smem_bytes;
+    int off_logits, off_xchg, off_wml, off_slots, off_misc, off_bars, smem_bytes;
 };
 
 struct DecodeArgs {

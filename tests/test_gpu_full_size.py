@@ -57,7 +57,7 @@ def test_config4_bench_launch_shape():
     inf = ls.eng.info()
     assert (inf.splits, inf.groups, inf.grid) == (1, 2, sms)
     if sms == 148:
-        assert (inf.stages, inf.tail_units, inf.tail_splits) == (6, 32, 4)
+        assert (inf.stages, inf.tail_units, inf.tail_splits) == (5, 32, 4)
 
 
 def test_config5_full_batch():

@@ -73,7 +73,7 @@ def test_softmax_reference_is_raised_late():
 
 
 @pytest.mark.parametrize("groups", [1, 2])
-@pytest.mark.parametrize("splits,stages", [(1, 2), (1, 3), (2, 3), (1, 5), (4, 2), (3, 4), (6, 6)])
+@pytest.mark.parametrize("splits,stages", [(1, 2), (1, 3), (2, 3), (1, 5), (4, 2), (3, 4), (6, 5)])
 def test_ring_depths_and_warp_groups(splits, stages, groups):
     """Shallow and odd ring depths with one and two groups of consumer warps: with two groups a
     stage's consecutive uses go to different groups, and a block's page count may be odd, so
