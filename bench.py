@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # 592-unit case of the same launch shape; traffic grows in proportion to units x tokens, so a full
 # launch is scaled by its algorithmic bytes.  Valid only for the kernel sources it was taken on.
 NCU_DECODE_CAPTURE = {
-    "traffic_per_algorithmic_byte": 1.0080,
-    "sha256": {"decode.cu": "cdadef6063986bfef98f17ef539659e9af82c5c6d780106325e27dbcf87a0519",
+    "traffic_per_algorithmic_byte": 1.0078,
+    "sha256": {"decode.cu": "6b84d5716e1614d3e322f8a3cd1df571ee01966570b3b7f03d4eac9679c5497d",
                "common.cuh": "e145966ccf290b94a07f9b5374ce552520833824b6b9440fc6aa85adf416adac"},
 }
 
