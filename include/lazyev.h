@@ -121,6 +121,24 @@ int lazyev_set_page_table(lazyev_t* h, const int32_t* host_table);
 int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens);
 
 /*
+ * Prompt load WITH observation.  The paper tracks recurrence while decoding and does not say
+ * how TS and MRI of prompt tokens start; lazyev_prefill() takes TS = 0, MRI = 0.  This call
+ * takes the other reading: tracking (Eq. 1, Algorithm 1's per-token loop) starts at the first
+ * prompt token.  The prompt is loaded and then replayed through the decode kernel one row at
+ * a time: row j attends causally over rows 0..j with its own queries, and the statistics are
+ * updated at time j - (n_tokens - 1), so the last prompt row is time 0 and decode steps
+ * continue at t = 1; a prompt token starts at TS = its own time, MRI = 0.  No eviction
+ * happens during the prompt.
+ *   q, out : [n_tokens][layers, batch, q_heads, head_dim] bf16 (row-major by prompt position:
+ *            row j is laid out like the q / out of lazyev_decode_step); out receives the
+ *            causal attention output of every prompt row
+ *   k, v   : as for lazyev_prefill()
+ * Cost: n_tokens decode launches over 1..n_tokens cached tokens (meant for prompts of
+ * hundreds to a few thousand tokens).  Errors as for lazyev_prefill().
+ */
+int lazyev_prefill_observed(lazyev_t* h, const void* q, const void* k, const void* v, int n_tokens, void* out);
+
+/*
  * One decode step for all units (Algorithm 1 without its last branch unless
  * automatic eviction is on):
  *   t += 1; the new token (k_new, v_new) is appended with TS = t, MRI = 0;

@@ -224,6 +224,31 @@ class OracleUnit:
         self.MRI = np.zeros(self.P, dtype=np.int64)
         self.t = 0
 
+    def prefill_observed(self, Q, K, V) -> np.ndarray:
+        """Prompt load with tracking from the first prompt token (the paper does not say how
+        TS / MRI of prompt tokens start; this is the reading in which Algorithm 1's per-token
+        loop already runs over the prompt).  Row j of the prompt attends causally over rows
+        0..j at time j - (P - 1), so the last row is time 0 and decode steps go on at t = 1.
+        Q [P, G, D], K, V [P, D].  Returns the attention outputs [P, G, D]."""
+        Q = np.asarray(Q, dtype=np.float64)
+        K = np.asarray(K, dtype=np.float64)
+        V = np.asarray(V, dtype=np.float64)
+        P = K.shape[0]
+        self.P = P
+        self.pos = np.zeros(0, dtype=np.int64)
+        self.K, self.V = np.zeros((0, self.D)), np.zeros((0, self.D))
+        self.TS, self.MRI = np.zeros(0, dtype=np.int64), np.zeros(0, dtype=np.int64)
+        self.t = -P                       # attend() advances t before it appends: row j runs at j - (P - 1)
+        outs = np.zeros((P, self.G, self.D))
+        self.prompt_margin = np.full(P, np.inf)      # per token: closest |pbar - alpha| / alpha over the rows
+        for j in range(P):
+            outs[j], pbar = self.attend(Q[j], K[j], V[j])
+            m = np.abs(pbar - float(self.alpha32)) / max(float(self.alpha32), 1e-300)
+            self.prompt_margin[: j + 1] = np.minimum(self.prompt_margin[: j + 1], m)
+            self.track(pbar)
+        assert self.t == 0 and self.n == P
+        return outs
+
     # -- one decode step --------------------------------------------------------
     def attend(self, q, k_new, v_new):
         """t += 1, append the new token, evaluate Eq. (attn).

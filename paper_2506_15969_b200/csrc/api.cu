@@ -1,4 +1,5 @@
 // C-ABI layer: host-side handle, argument validation, step / eviction schedule, launches.
+#include <limits.h>
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
@@ -251,18 +252,10 @@ struct HostPipe {
     uint8_t* out_host;
 };
 
-int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out, const HostPipe* pipe = nullptr) {
-    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
-    if (h->n + 1 > h->capacity) return fail(h, LAZYEV_ECAPACITY, "cache full (%d slots per unit)", h->capacity);
-    const Geometry geo = geometry(h);
-    const int t = h->t + 1, n = h->n + 1;
-    cudaError_t e;
-    {
-        SpanGuard g(h, kSpanAppend, 0.0);
-        e = append_launch(geo, h->pool, h->st, k_new, v_new, n - 1, t, h->prefill + t - 1, h->stream);
-    }
-    if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
-
+// The decode launches of one step: attention of q over the first n cached tokens of every unit with
+// tracking at time t.
+int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPipe* pipe) {
+    cudaError_t e = cudaSuccess;
     DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages, h->force_groups};
     // Launch shape, chosen per number of pages in use and cached.  Every cluster size whose logits fit
     // gets a relative speed (blocks per unit, discounted for the per-unit exchange between the blocks
@@ -378,11 +371,26 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
         }
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "decode kernel launch");
-    h->launches += 1;      // the append kernel
     h->last_plan = plan;
     h->last_tail_units = shape.tail_units;
     h->last_tail_splits = shape.tail_splits;
     h->last_grid = clusters * plan.splits;
+    return LAZYEV_OK;
+}
+
+int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out, const HostPipe* pipe = nullptr) {
+    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
+    if (h->n + 1 > h->capacity) return fail(h, LAZYEV_ECAPACITY, "cache full (%d slots per unit)", h->capacity);
+    const int t = h->t + 1, n = h->n + 1;
+    cudaError_t e;
+    {
+        SpanGuard g(h, kSpanAppend, 0.0);
+        e = append_launch(geometry(h), h->pool, h->st, k_new, v_new, n - 1, t, h->prefill + t - 1, h->stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
+    h->launches += 1;
+    const int rc = run_decode(h, q, out, n, t, pipe);
+    if (rc != LAZYEV_OK) return rc;
     h->t = t;
     h->n = n;
     if (h->auto_evict) return run_evict(h, nullptr);
@@ -580,9 +588,32 @@ int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens) {
     if (h->prefilled) return fail(h, LAZYEV_ESTATE, "prefill called twice");
     if (!k || !v || n_tokens <= 0) return fail(h, LAZYEV_EINVAL, "null pointer or non-positive token count");
     if (n_tokens > h->max_prefill) return fail(h, LAZYEV_ECAPACITY, "prompt of %d tokens exceeds max_prefill = %d", n_tokens, h->max_prefill);
-    cudaError_t e = prefill_launch(geometry(h), h->pool, h->st, k, v, n_tokens, h->stream);
+    cudaError_t e = prefill_launch(geometry(h), h->pool, h->st, k, v, n_tokens, INT_MIN, h->stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "prefill kernel launch");
     h->launches += 1;
+    h->prefilled = true;
+    h->prefill = n_tokens;
+    h->n = n_tokens;
+    h->t = 0;
+    return LAZYEV_OK;
+}
+
+int lazyev_prefill_observed(lazyev_t* h, const void* q, const void* k, const void* v, int n_tokens, void* out) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "prefill before bind");
+    if (h->prefilled) return fail(h, LAZYEV_ESTATE, "prefill called twice");
+    if (!q || !k || !v || !out || n_tokens <= 0) return fail(h, LAZYEV_EINVAL, "null pointer or non-positive token count");
+    if (n_tokens > h->max_prefill) return fail(h, LAZYEV_ECAPACITY, "prompt of %d tokens exceeds max_prefill = %d", n_tokens, h->max_prefill);
+    // rows are loaded with TS = their own time j - (P - 1) <= 0, then replayed through the decode kernel
+    cudaError_t e = prefill_launch(geometry(h), h->pool, h->st, k, v, n_tokens, 1 - n_tokens, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "prefill kernel launch");
+    h->launches += 1;
+    const size_t row_bytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
+    for (int j = 0; j < n_tokens; ++j) {
+        const int rc = run_decode(h, (const uint8_t*)q + j * row_bytes, (uint8_t*)out + j * row_bytes, j + 1,
+                                  j - (n_tokens - 1), nullptr);
+        if (rc != LAZYEV_OK) return rc;
+    }
     h->prefilled = true;
     h->prefill = n_tokens;
     h->n = n_tokens;

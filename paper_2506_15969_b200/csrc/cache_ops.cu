@@ -1,4 +1,6 @@
 // Cache maintenance kernels: state initialisation, prompt load, per-step append.
+#include <limits.h>
+
 #include "internal.h"
 
 namespace lzk {
@@ -21,7 +23,7 @@ __global__ void init_state_kernel(Geometry geo, StateView st) {
 
 // One warp per (unit, token): lanes 0..15 move the K row's chunks, lanes 16..31 the V row's.
 __global__ void prefill_kernel(Geometry geo, uint8_t* pool, StateView st, const uint4* __restrict__ k,
-                               const uint4* __restrict__ v, int n_tokens) {
+                               const uint4* __restrict__ v, int n_tokens, int ts_first) {
     const int lane = threadIdx.x & 31;
     const size_t warps = ((size_t)gridDim.x * blockDim.x) >> 5;
     const size_t total = (size_t)geo.units * n_tokens;
@@ -34,7 +36,9 @@ __global__ void prefill_kernel(Geometry geo, uint8_t* pool, StateView st, const 
         *reinterpret_cast<uint4*>(row + swz_chunk(c, r) * 16) = *src;
         if (lane == 0) {
             const size_t s = (size_t)u * geo.capacity + i;
-            st.ts[s] = 0;          // prompt tokens start at TS = 0, MRI = 0 (Section 4: MRI starts at 0)
+            // Prompt tokens start at MRI = 0 (Section 4) and TS = 0, or, when the prompt is going to be
+            // replayed with tracking, at their own time ts_first + i (the last prompt row is time 0).
+            st.ts[s] = ts_first == INT_MIN ? 0 : ts_first + i;
             st.mri[s] = 0;
             st.pos[s] = i;
         }
@@ -68,11 +72,11 @@ cudaError_t init_state_launch(const Geometry& geo, StateView st, cudaStream_t st
 }
 
 cudaError_t prefill_launch(const Geometry& geo, uint8_t* pool, StateView st, const void* k, const void* v,
-                           int n_tokens, cudaStream_t stream) {
+                           int n_tokens, int ts_first, cudaStream_t stream) {
     const size_t rows = (size_t)geo.units * n_tokens;
     const int blocks = (int)((rows + 7) / 8 < 148 * 16 ? (rows + 7) / 8 : 148 * 16);
     prefill_kernel<<<blocks, 256, 0, stream>>>(geo, pool, st, reinterpret_cast<const uint4*>(k),
-                                               reinterpret_cast<const uint4*>(v), n_tokens);
+                                               reinterpret_cast<const uint4*>(v), n_tokens, ts_first);
     return cudaGetLastError();
 }
 

@@ -39,8 +39,9 @@ cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clu
 
 // ---- cache maintenance ---------------------------------------------------------
 cudaError_t init_state_launch(const Geometry& geo, StateView st, cudaStream_t stream);
+// ts_first = INT_MIN: every prompt token starts at TS = 0; otherwise token i starts at TS = ts_first + i.
 cudaError_t prefill_launch(const Geometry& geo, uint8_t* pool, StateView st, const void* k, const void* v,
-                           int n_tokens, cudaStream_t stream);
+                           int n_tokens, int ts_first, cudaStream_t stream);
 cudaError_t append_launch(const Geometry& geo, uint8_t* pool, StateView st, const void* k_new, const void* v_new,
                           int slot, int t, int position, cudaStream_t stream);
 

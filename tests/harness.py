@@ -56,7 +56,7 @@ def make_oracle(cfg: traces.TraceConfig, score_mode="h1+h2") -> orc.OracleUnit:
 class Lockstep:
     def __init__(self, cfg: traces.TraceConfig, seed: int, sample_units, splits: int = 0, stages: int = 0,
                  score_mode: int = 0, page_table=None, pure: bool = True, check_inputs: bool = True,
-                 groups: int = 0):
+                 groups: int = 0, observed: bool = False):
         self.cfg, self.sample = cfg, list(sample_units)
         self.eng = make_engine(cfg)
         self.eng.set_auto_evict(False)
@@ -83,13 +83,53 @@ class Lockstep:
         kc, vc = self.gen_cpu.prefill()
         if check_inputs:
             assert torch.equal(k[self.sample].cpu(), kc) and torch.equal(v[self.sample].cpu(), vc)
-        self.eng.prefill(k.view(L, Bt, cfg.kv_heads, cfg.prefill, cfg.head_dim),
-                         v.view(L, Bt, cfg.kv_heads, cfg.prefill, cfg.head_dim))
-        for i in range(len(self.sample)):
-            self.shadow[i].prefill(f64(kc[i]), f64(vc[i]))
-            if self.pure:
-                self.pure[i].prefill(f64(kc[i]), f64(vc[i]))
+        kk = k.view(L, Bt, cfg.kv_heads, cfg.prefill, cfg.head_dim)
+        vv = v.view(L, Bt, cfg.kv_heads, cfg.prefill, cfg.head_dim)
+        if not observed:
+            self.eng.prefill(kk, vv)
+            for i in range(len(self.sample)):
+                self.shadow[i].prefill(f64(kc[i]), f64(vc[i]))
+                if self.pure:
+                    self.pure[i].prefill(f64(kc[i]), f64(vc[i]))
+        else:
+            self._observed_prefill(kk, vv, kc, vc, seed)
         self.t = 0
+
+    def _observed_prefill(self, kk, vv, kc, vc, seed):
+        """Prompt load with tracking: seeded prompt queries, some rows re-aligned with earlier keys so
+        that prompt tokens are re-activated; GPU against the oracle, then the shadow adopts the GPU's
+        TS / MRI (they may differ only where a probability came within 1e-4 (relative) of the threshold)."""
+        cfg, P = self.cfg, self.cfg.prefill
+        g = torch.Generator().manual_seed(1000 + seed)
+        q = torch.randn(P, cfg.units, cfg.group, cfg.head_dim, generator=g)
+        kf = kk.reshape(cfg.units, P, cfg.head_dim).float().cpu()
+        rows = torch.randint(1, P, (cfg.units, P // 6), generator=g)
+        for u in range(cfg.units):
+            for j in rows[u].tolist():
+                i = int(torch.randint(0, j, (1,), generator=g))
+                q[j, u] += 4.0 * (cfg.head_dim ** 0.5) * kf[u, i] / kf[u, i].pow(2).sum()
+        q = q.to(torch.bfloat16)
+        out = torch.empty(P, cfg.units, cfg.group, cfg.head_dim, dtype=torch.bfloat16, device="cuda")
+        self.eng.prefill_observed(q.cuda(), kk, vv, out)
+        rep = self.rep
+        self.prompt_excluded = 0
+        for i, u in enumerate(self.sample):
+            sh = self.shadow[i]
+            ref = sh.prefill_observed(f64(q[:, u]), f64(kc[i]), f64(vc[i]))
+            if self.pure:
+                self.pure[i].prefill_observed(f64(q[:, u]), f64(kc[i]), f64(vc[i]))
+            got = f64(out[:, u])
+            rep.max_out_err = max(rep.max_out_err, float((np.abs(got - ref) / (OUT_ATOL + OUT_RTOL * np.abs(ref))).max()))
+            d = self._dump(u)
+            assert d["n"] == P and d["t"] == 0
+            rep.max_pbar_err = max(rep.max_pbar_err, float(np.abs(d["pbar"][0] - sh.last_pbar).max()))
+            clear = sh.prompt_margin > 1e-4
+            assert np.array_equal(d["ts"][0][clear], sh.TS[clear]), f"prompt TS mismatch unit {u}"
+            assert np.array_equal(d["mri"][0][clear], sh.MRI[clear]), f"prompt MRI mismatch unit {u}"
+            assert np.array_equal(d["pos"][0], sh.pos)
+            self.prompt_excluded += int((~clear).sum())
+            rep.activations += int((sh.MRI > 0).sum())
+            sh.TS, sh.MRI = d["ts"][0].astype(np.int64), d["mri"][0].astype(np.int64)
 
     def _dump(self, u, **kw):
         return self.eng.dump_state(u, 1, **kw)

@@ -238,6 +238,21 @@ def test_mri_histogram_and_quantile_match_the_oracle():
         ls.eng.mri_histogram(16, 7, 2)
 
 
+@pytest.mark.parametrize("prefill", [150, 333])
+def test_observed_prompt_then_decode(prefill):
+    """lazyev_prefill_observed: causal prompt attention row by row with tracking from the first
+    token, against the oracle; then decoding with evictions continues in lock step."""
+    cfg = traces.tiny_config(prefill=prefill, budget=prefill + 40, window=32, alpha=0.02)
+    ls = lockstep(cfg, seed=17, sample_units=[0, 3, 6], observed=True)
+    d = ls.eng.dump_state(0, 1)
+    assert (d["ts"][0] >= np.arange(prefill) - (prefill - 1)).all() and d["ts"][0].max() == 0
+    assert (d["mri"][0] > 0).sum() >= 5                       # prompt tokens were re-activated
+    assert ls.prompt_excluded <= prefill // 25                # tokens that came within 1e-4 of the threshold
+    rep = ls.run(100)
+    ls.assert_ok(jaccard=0.98)
+    assert rep.evictions == 2
+
+
 def test_resume_from_a_snapshot_continues_bit_for_bit():
     """dump_state -> load_state into a fresh handle (with a larger capacity): the resumed run must
     produce the same outputs, statistics, evictions and cache as the run that was never stopped."""

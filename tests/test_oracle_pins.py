@@ -255,6 +255,36 @@ def test_decreasing_h2_variant_has_the_properties_the_appendix_requires():
     assert I(3, 3) > I(30, 30) and float(orc.importance(100, 97, 3)) < float(orc.importance(100, 70, 30))
 
 
+def test_observed_prompt_is_causal_attention_with_tracking_from_the_first_token():
+    """Outputs equal the library's causal SDPA; with alpha > 1 nothing is re-activated and every
+    token keeps TS = its own time j - (P - 1); a planted key re-activated at known rows gets
+    the hand-computed TS and MRI; decode steps continue at t = 1."""
+    rng = np.random.default_rng(11)
+    P, G, D = 37, 3, 16
+    Q, K, V = rng.standard_normal((P, G, D)), rng.standard_normal((P, D)), rng.standard_normal((P, D))
+    o = orc.OracleUnit(G, D, 100, 8, 1.5)
+    outs = o.prefill_observed(Q, K, V)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q).permute(1, 0, 2)[None], torch.from_numpy(K)[None, None].expand(1, G, P, D),
+        torch.from_numpy(V)[None, None].expand(1, G, P, D), is_causal=True)[0].permute(1, 0, 2).numpy()
+    assert np.abs(outs - ref).max() < 1e-12
+    assert o.TS.tolist() == [j - (P - 1) for j in range(P)] and not o.MRI.any()
+    assert o.pos.tolist() == list(range(P)) and o.t == 0
+    # token 2 is made to dominate rows 5, 9 and 20 (and is active at its own row 2): gaps 3, 4, 11
+    K2, Q2 = 0.01 * rng.standard_normal((P, D)), 0.01 * rng.standard_normal((P, G, D))
+    K2[2] = 0.0; K2[2, 0] = 8.0
+    for j in (5, 9, 20):
+        Q2[j, :, 0] = 8.0
+    o2 = orc.OracleUnit(G, D, 100, 8, 0.6)
+    o2.prefill_observed(Q2, K2, V)
+    assert o2.TS[2] == 20 - (P - 1) and o2.MRI[2] == 11
+    # every token is active at its own row only when it takes >= 0.6 of the weight: row 0 always does
+    assert o2.TS[0] == 0 - (P - 1) and o2.MRI[0] == 0
+    _, pbar = o2.attend(Q2[5], K2[3], V[3])                  # first decode step: t = 1, position P
+    o2.track(pbar)
+    assert o2.t == 1 and o2.pos[-1] == P and o2.TS[2] == 1 and o2.MRI[2] == 1 - (20 - (P - 1))
+
+
 def test_mri_histogram_and_quantile_closed_forms_and_library_routine():
     """One token per MRI value 1..100 (plus never re-activated ones): the 80 % value is 80;
     on random data the rule equals numpy's inverted-CDF percentile of the re-activated tokens."""
