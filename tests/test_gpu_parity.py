@@ -217,6 +217,32 @@ def test_per_step_eviction_window_of_one():
     assert ls.rep.evictions == 90 - 20 and ls.eng.info().n == 120
 
 
+@pytest.mark.parametrize("case", range(24))
+def test_random_shapes_and_launch_shapes(case):
+    """Seeded random combinations of group size, unit count, cache length, window, protection and
+    forced launch shapes (cluster size, ring depth, warp groups), a few windows each."""
+    rng = np.random.default_rng(1000 + case)
+    kv_heads = int(rng.integers(1, 4))
+    group = int(rng.integers(1, 9))
+    batch, layers = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    window = int(rng.choice([8, 16, 32, 48]))
+    n_recent = int(rng.integers(1, window + 1))
+    n_initial = int(rng.integers(0, 5))
+    prefill = int(rng.integers(1, 700))
+    budget = max(n_recent + n_initial + 2, window + 1, int(prefill * rng.uniform(0.5, 1.3)))
+    splits = int(rng.choice([0, 0, 1, 2, 3, 5, 8]))
+    groups = int(rng.choice([0, 1, 2]))
+    stages = int(rng.choice([0, 0, 2, 3, 4, 5]))
+    cfg = traces.tiny_config(batch=batch, layers=layers, q_heads=group * kv_heads, kv_heads=kv_heads, prefill=prefill,
+                             budget=budget, window=window, n_recent=n_recent, n_initial=n_initial,
+                             alpha=float(rng.choice([0.0, 0.003, 0.02])), period_lo=40, period_hi=120)
+    units = sorted(set(int(x) for x in rng.integers(0, cfg.units, size=3)))
+    ls = lockstep(cfg, seed=case, sample_units=units, splits=splits, stages=stages, groups=groups, pure=False)
+    rep = ls.run(3 * window + 5)
+    ls.assert_ok()
+    assert rep.steps == 3 * window + 5 and ls.eng.dump_state(0, 1)["device_status"] == 0
+
+
 def test_mri_histogram_and_quantile_match_the_oracle():
     """The live distribution of MRI (the paper's offline rule for choosing W): bit-exact counts."""
     from oracle import lazyev_oracle as orc
