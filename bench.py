@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # launch is scaled by its algorithmic bytes.  Valid only for the kernel sources it was taken on.
 NCU_DECODE_CAPTURE = {
     "traffic_per_algorithmic_byte": 1.0078,
-    "sha256": {"decode.cu": "6b84d5716e1614d3e322f8a3cd1df571ee01966570b3b7f03d4eac9679c5497d",
+    "sha256": {"decode.cu": "48f834a620d16014efd666520e124e8812a10d4ed675eee409174a7042e1737b",
                "common.cuh": "e145966ccf290b94a07f9b5374ce552520833824b6b9440fc6aa85adf416adac"},
 }
 

@@ -6,26 +6,29 @@
 // and, fused (Section 4 "Recurrence Interval Tracking", Eq. (1), Algorithm 1):
 //   pbar[i] = mean_g p_g[i];  if pbar[i] >= alpha: MRI[i] = max(MRI[i], t - TS[i]); TS[i] = t.
 //
-// Structure: persistent blocks, one block per SM, grouped in clusters of
-// `splits` blocks.  A cluster walks units round-robin; its blocks split the
-// unit's pages.  Inside a block one producer warp streams 32 KiB pages into a
-// shared-memory ring with linear bulk copies (TMA engine, mbarrier completion).
-// Consumer warps come in groups of four; a group takes a whole page, 16 tokens
-// per warp, and with two groups consecutive pages are worked on concurrently.
+// Structure: persistent blocks, one block per SM.  A block -- or, when a unit's
+// logits do not fit one SM, a cluster of `splits` blocks that split the unit's
+// pages -- walks units round-robin.  Inside a block one producer warp streams
+// 32 KiB pages into a shared-memory ring with linear bulk copies (TMA engine,
+// mbarrier completion).  Consumer warps come in groups of four; a group takes a
+// whole page, 16 tokens per warp, and with two groups consecutive pages are
+// worked on concurrently.
 //
 // Per 16 tokens a warp runs S^T = K Q^T (tokens are the M rows, query heads the
 // N columns) and O^T += V^T P^T (head dimensions are the M rows) on mma.sync
 // m16n8k16, so both operands that come from the cache fill the whole A tile and
 // the eight query-head columns fill the N = 8 tile.  P goes from the accumulator
-// layout of the first product to the B layout of the second with two movmatrix
-// transposes.  Softmax is online against a per-warp, per-head reference value
-// that is raised (and O, l rescaled) only when a logit exceeds it by more than
-// 2^8, found with one warp vote per tile; any reference gives the same sums.
+// layout of the first product to the B layout of the second with movmatrix
+// transposes, as two bf16 terms (hi + lo).  Softmax is online against a per-warp,
+// per-head reference value that is raised (and O, l rescaled) only when a logit
+// exceeds it by more than 2^8, found with one warp vote per tile; any reference
+// gives the same sums.
 //
 // The scaled logits of the block's chunk stay on chip: in tensor memory (TMEM,
 // used as 512 private 32-bit words per consumer thread through tcgen05.ld / st),
-// and in shared memory for the pages beyond the 128 that fit there.  After the chunk the warps and then the cluster's blocks
-// merge (reference, l, O) through (distributed) shared memory, which gives the
+// and in shared memory for the pages beyond the 128 that fit there.  After the
+// chunk the warps merge (reference, l, O) through per-warp shared-memory slots
+// and the cluster's blocks through distributed shared memory, which gives the
 // exact log-sum-exp.  The probabilities of a unit are produced while the block's
 // NEXT unit streams: the warp that is about to overwrite the logits of a
 // 16-token tile first turns the old ones into pbar, writes it and updates
