@@ -169,6 +169,9 @@ int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const
  * the front of each unit in generation order; n becomes budget_now.
  * Otherwise does nothing and returns 0.  `*evicted` (optional) receives the
  * number of tokens removed per unit.
+ * Limit: the selection keeps one 64-bit key per unprotected token in shared memory, so an
+ * eviction over more than 25 600 unprotected tokens per unit returns EINVAL and changes
+ * nothing (a cache that never evicts may be longer).  Other errors: ESTATE (no prefill), ECUDA.
  */
 int lazyev_evict(lazyev_t* h, int* evicted);
 

@@ -347,6 +347,23 @@ def test_call_order_errors_and_capacity():
     assert eng.dump_state()["device_status"] == 0
 
 
+def test_eviction_over_too_many_candidates_is_refused():
+    """More than 25 600 unprotected tokens per unit: lazyev_evict says so and leaves the cache alone."""
+    eng = binding.Engine(1, 2, 1, 128, 25700, 64, 0.5, max_prefill=25700)
+    z = torch.zeros(1, 1, 1, 25700, 128, dtype=torch.bfloat16, device="cuda")
+    eng.prefill(z, z)
+    eng.set_auto_evict(False)
+    x = torch.zeros(1, 1, 2, 128, dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros(1, 1, 1, 128, dtype=torch.bfloat16, device="cuda")
+    for _ in range(64):
+        eng.decode_step(x, kv, kv, x)
+    with pytest.raises(binding.LazyEvError) as e:
+        eng.evict()
+    assert e.value.code == binding.EINVAL and "candidates" in str(e.value)
+    eng.synchronize()
+    assert eng.info().n == 25764 and eng.dump_state()["device_status"] == 0
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     cfg = traces.tiny_config()
     gen = traces.TraceGen(cfg, 8, device="cuda")
