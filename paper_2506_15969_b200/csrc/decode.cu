@@ -272,6 +272,23 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
 
         // pbar, TS and MRI of tokens (base + g) and (base + g + 8) of the previous unit from its logits
         // (base: token index inside the block's chunk).
+        // Eq. (1) for an activated token needs its old TS.  The load is issued when the activation is
+        // found and its result is used one emit_previous call later (a page's worth of work), so the
+        // update never stalls the warp that holds a ring stage; at most one token per half is pending.
+        long long pend_idx0 = -1, pend_idx1 = -1;
+        int32_t pend_ts0 = 0, pend_ts1 = 0;
+        auto retire_pending = [&]() {
+            if (pend_idx0 >= 0) {
+                atomicMax(&p.mri[pend_idx0], p.t - pend_ts0);      // MRI = max(MRI, t - TS)
+                p.ts[pend_idx0] = p.t;                             // TS = t
+                pend_idx0 = -1;
+            }
+            if (pend_idx1 >= 0) {
+                atomicMax(&p.mri[pend_idx1], p.t - pend_ts1);
+                p.ts[pend_idx1] = p.t;
+                pend_idx1 = -1;
+            }
+        };
         auto emit_previous = [&](int base, float x00, float x01, float x10, float x11) {
             float a0 = h0_on ? fast_exp2(x00 - lse0) : 0.f;
             float a1 = h0_on ? fast_exp2(x10 - lse0) : 0.f;
@@ -284,18 +301,23 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
             a0 += __shfl_xor_sync(0xffffffffu, a0, 2);
             a1 += __shfl_xor_sync(0xffffffffu, a1, 2);
             if (qd == 0) {
+                retire_pending();
                 const size_t row = (size_t)u_prev * p.capacity + tok0;
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const int i = base + g + 8 * half;
-                    if (tok0 + i < p.n) {
-                        const float pb = (half ? a1 : a0) * p.inv_group;
-                        p.pbar[row + i] = pb;
-                        if (pb >= p.alpha) {
-                            const int32_t gap = p.t - p.ts[row + i];
-                            if (gap > p.mri[row + i]) p.mri[row + i] = gap;
-                            p.ts[row + i] = p.t;
-                        }
+                const int i0 = base + g, i1 = base + g + 8;
+                if (tok0 + i0 < p.n) {
+                    const float pb = a0 * p.inv_group;
+                    p.pbar[row + i0] = pb;
+                    if (pb >= p.alpha) {
+                        pend_idx0 = (long long)(row + i0);
+                        pend_ts0 = p.ts[row + i0];
+                    }
+                }
+                if (tok0 + i1 < p.n) {
+                    const float pb = a1 * p.inv_group;
+                    p.pbar[row + i1] = pb;
+                    if (pb >= p.alpha) {
+                        pend_idx1 = (long long)(row + i1);
+                        pend_ts1 = p.ts[row + i1];
                     }
                 }
             }
@@ -531,6 +553,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 emit_previous(j * kPageTokens + (int)tok_off, y00, y01, y10, y11);
             }
         }
+        retire_pending();
     }
 
     // No block may exit while a peer can still read its shared memory; tensor memory goes back last.
