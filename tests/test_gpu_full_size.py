@@ -64,3 +64,15 @@ def test_config5_full_batch():
     cfg = _steady(traces.CONFIGS[5], traces.CONFIGS[5].budget)          # 12288 units, 4915 + 1..256 tokens
     ls = _run(cfg, [0, 147, 6000, cfg.units - 4, cfg.units - 1], 2 * cfg.window + 2, 1, 2)
     assert ls.eng.info().n == cfg.budget + 2
+
+
+def test_config2_whole_trace_end_to_end():
+    """Configuration 2 from its 512-token prompt through all 4096 decode steps (20 evictions): every step
+    of two units in lock step with the oracle, and the kept sets of a pure-oracle run at the end."""
+    from tests.harness import Lockstep
+    cfg = traces.CONFIGS[2]
+    ls = Lockstep(cfg, seed=0, sample_units=[5, 42])
+    rep = ls.run(cfg.steps, check_every=4)
+    ls.assert_ok()
+    assert rep.evictions == (cfg.steps - 1664) // cfg.window + 1 and ls.eng.info().n == cfg.budget
+    assert rep.near_tie_events == 0 and rep.min_jaccard >= 0.999
