@@ -168,6 +168,11 @@ def _oracle_worker(job):
     import numpy as np
     import torch
     torch.set_num_threads(1)
+    try:                                     # one thread per worker, so that `cores` is what was really used
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(1)
+    except Exception:
+        pass
     from oracle import lazyev_oracle as orc
     from paper_2506_15969_b200 import traces
     cfg, seed, unit, n0, steps, warm = job
