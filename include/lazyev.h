@@ -121,6 +121,16 @@ int lazyev_set_page_table(lazyev_t* h, const int32_t* host_table);
 int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens);
 
 /*
+ * Forget the cached sequences and make the handle ready for a new prompt (lazyev_prefill,
+ * lazyev_prefill_observed or lazyev_load_state) on the same memory, configuration and stream:
+ * t and n return to 0, budget_now to the create-time budget, the device status word is
+ * cleared; the page table is kept.  Asynchronous on the bound stream.  (The paper processes
+ * one generation at a time; a server reuses the cache memory for the next batch of requests.)
+ * Errors: ESTATE (not bound), ECUDA.
+ */
+int lazyev_reset(lazyev_t* h);
+
+/*
  * Prompt load WITH observation.  The paper tracks recurrence while decoding and does not say
  * how TS and MRI of prompt tokens start; lazyev_prefill() takes TS = 0, MRI = 0.  This call
  * takes the other reading: tracking (Eq. 1, Algorithm 1's per-token loop) starts at the first

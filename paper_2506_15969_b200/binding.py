@@ -55,6 +55,7 @@ _PROTOS = {
     "lazyev_bind": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_set_page_table": [C.c_void_p, C.c_void_p],
     "lazyev_prefill": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int],
+    "lazyev_reset": [C.c_void_p],
     "lazyev_prefill_observed": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p],
     "lazyev_decode_step": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_decode_step_host": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
@@ -174,6 +175,9 @@ class Engine:
 
     def prefill(self, k, v) -> None:
         self._check(lib().lazyev_prefill(self._h, _ptr(k), _ptr(v), k.shape[-2]))
+
+    def reset(self) -> None:
+        self._check(lib().lazyev_reset(self._h))
 
     def prefill_observed(self, q, k, v, out) -> None:
         """lazyev_prefill_observed: q, out [P, layers, batch, q_heads, D]; k, v as for prefill."""

@@ -598,6 +598,19 @@ int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens) {
     return LAZYEV_OK;
 }
 
+int lazyev_reset(lazyev_t* h) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "reset before bind");
+    // Old rows stay in the pool: slots past n are masked, they only have to be finite.  The state arrays
+    // are rewritten by the next prompt load and by every append; the device status word is cleared.
+    cudaError_t e = cudaMemsetAsync(h->st.status, 0, 64, h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "clearing the device status word");
+    h->prefilled = false;
+    h->t = h->n = h->prefill = 0;
+    h->budget_now = h->budget;
+    return LAZYEV_OK;
+}
+
 int lazyev_prefill_observed(lazyev_t* h, const void* q, const void* k, const void* v, int n_tokens, void* out) {
     if (!h) return LAZYEV_EINVAL;
     if (!h->bound) return fail(h, LAZYEV_ESTATE, "prefill before bind");

@@ -279,6 +279,40 @@ def test_observed_prompt_then_decode(prefill):
     assert rep.evictions == 2
 
 
+def test_reset_then_a_new_sequence_gives_the_same_results_as_a_fresh_handle():
+    """A handle that served one batch of sequences is reset and serves another: outputs, statistics
+    and cache are those of a freshly created handle (nothing of the first batch leaks through)."""
+    from tests.harness import make_engine
+    cfg = traces.tiny_config()
+    shape = (cfg.layers, cfg.batch, cfg.kv_heads, cfg.prefill, 128)
+    used, fresh = make_engine(cfg), make_engine(cfg)
+    out_u = torch.empty(cfg.layers, cfg.batch, cfg.q_heads, 128, dtype=torch.bfloat16, device="cuda")
+    out_f = torch.empty_like(out_u)
+    first = traces.TraceGen(cfg, 30, device="cuda")
+    k, v = first.prefill()
+    used.prefill(k.view(shape), v.view(shape))
+    for _ in range(5):
+        q, kn, vn = first.steps(32)
+        for s in range(32):
+            used.decode_step(q[s], kn[s], vn[s], out_u)
+    assert used.info().evictions == 3
+    used.reset()
+    assert (used.info().t, used.info().n) == (0, 0)
+    second = traces.TraceGen(cfg, 31, device="cuda")
+    k, v = second.prefill()
+    used.prefill(k.view(shape), v.view(shape)); fresh.prefill(k.view(shape), v.view(shape))
+    for _ in range(4):
+        q, kn, vn = second.steps(32)
+        for s in range(32):
+            used.decode_step(q[s], kn[s], vn[s], out_u)
+            fresh.decode_step(q[s], kn[s], vn[s], out_f)
+            assert torch.equal(out_u, out_f)
+    du, df = used.dump_state(kv=True), fresh.dump_state(kv=True)
+    for key in ("pos", "ts", "mri", "pbar", "k", "v"):
+        assert np.array_equal(du[key], df[key]), key
+    assert du["n"] == df["n"] == cfg.budget + 0 and du["device_status"] == 0
+
+
 def test_resume_from_a_snapshot_continues_bit_for_bit():
     """dump_state -> load_state into a fresh handle (with a larger capacity): the resumed run must
     produce the same outputs, statistics, evictions and cache as the run that was never stopped."""
