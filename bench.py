@@ -221,7 +221,7 @@ def run_reference(args):
     cores = os.cpu_count() or 1
     units = list(range(0, cfg.units, max(1, cfg.units // cores)))[:cores]
     n0 = cfg.budget
-    steps = max(1, min(args.steps, 24))
+    steps = max(1, min(args.steps, 128))
     tps, used, sample, ms = time_oracle(cfg, args.seed, units, n0, steps, min(args.warmup, 3))
     line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": cfg.batch / tps * 1e3,
@@ -371,8 +371,8 @@ def run_ours(args):
         cores = os.cpu_count() or 1
         n_units = args.cpu_units or cores
         sample_units = list(range(0, cfg.units, max(1, cfg.units // n_units)))[:n_units]
-        per_step_est = 6e-6 * inf.n * cfg.group / 7 + 2e-4          # seconds per unit-step, rough
-        steps_cpu = args.cpu_steps or int(max(4, min(16, 2.0 / max(per_step_est, 1e-6))))
+        per_step_est = 1.0e-6 * inf.n * cfg.group / 7 + 2e-4        # seconds per unit-step on one core, rough
+        steps_cpu = args.cpu_steps or int(max(8, min(128, 1.0 / max(per_step_est, 1e-6))))
         tps, used, sample, _ = time_oracle(cfg, args.seed, sample_units, inf.budget_now, steps_cpu, 2)
         cpu = {"value": tps, "unit": "tokens/s", "cores": used, "kind": "oracle", "sample": sample}
 
