@@ -15,7 +15,7 @@
 
 using namespace lzk;
 
-constexpr int kHostChunks = 4;            // unit ranges the host-buffer entry point pipelines copies over
+constexpr int kHostChunks = 3;            // unit ranges the host-buffer entry point pipelines copies over
 
 struct lazyev {
     // configuration
@@ -333,11 +333,15 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
         // rounds so that copies of one range overlap the kernel of another; then the last round's units.
         int begin[kHostChunks + 1], count[kHostChunks + 1], ranges = 0;
         const int rounds = (main_units + clusters - 1) / clusters;
-        const int parts = pipe ? (rounds < kHostChunks ? rounds : kHostChunks) : 1;
+        // (short first and last ranges: the first query copy and the last output copy are not overlapped)
+        static const int kShare[kHostChunks + 1] = {0, 1, 11, 12};       // cumulative twelfths of the rounds
+        const bool split = pipe && rounds >= 12;
+        const int parts = split ? kHostChunks : 1;
         for (int r = 0; r < parts; ++r) {
-            const int b = (int)((long long)rounds * r / parts) * clusters;
-            int e2 = (int)((long long)rounds * (r + 1) / parts) * clusters;
+            const int b = split ? rounds * kShare[r] / 12 * clusters : 0;
+            int e2 = split ? rounds * kShare[r + 1] / 12 * clusters : main_units;
             if (e2 > main_units) e2 = main_units;
+            if (e2 <= b) continue;
             begin[ranges] = b;
             count[ranges++] = e2 - b;
         }
