@@ -40,6 +40,9 @@ struct lazyev {
     unsigned long long* stage_hist = nullptr;
     // host-buffer entry point: copy streams and events, created at its first call
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    // second launch of a step (the partly filled last round) runs beside the end of the main launch
+    cudaStream_t tail_stream = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaEvent_t ev_in[kHostChunks + 1] = {}, ev_done[kHostChunks + 1] = {}, ev_ready = nullptr;
     // progress
     int t = 0, n = 0, prefill = 0;
@@ -357,14 +360,35 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
                 if (e == cudaSuccess) e = cudaEventRecord(h->ev_in[r], h->copy_in);
             }
         }
+        // The last round's units do not depend on the main launch: on a lower-priority stream of their own,
+        // forked here (after the append), their blocks take the SMs that the main launch's blocks leave as
+        // they finish; the bound stream joins afterwards.
+        const bool fork = shape.tail_units > 0 && !pipe && ranges > 1;
+        if (fork) {
+            if (!h->tail_stream) {
+                int lo = 0, hi = 0;
+                e = cudaDeviceGetStreamPriorityRange(&lo, &hi);
+                if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->tail_stream, cudaStreamNonBlocking, lo);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+                if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+            }
+            if (e == cudaSuccess) e = cudaEventRecord(h->ev_fork, h->stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(h->tail_stream, h->ev_fork, 0);
+        }
         for (int r = 0; r < ranges && e == cudaSuccess; ++r) {
             const bool is_tail = shape.tail_units > 0 && r == ranges - 1;
             if (pipe) e = cudaStreamWaitEvent(h->stream, h->ev_in[r], 0);
             if (e != cudaSuccess) break;
             DecodeArgs a{h->pool, h->st, q, out, n, t, begin[r], count[r]};
+            const bool beside = is_tail && fork;
+            if (e != cudaSuccess) break;
             e = decode_launch(c, is_tail ? tail_plan : plan, is_tail ? count[r] : (clusters < count[r] ? clusters : count[r]), a,
-                              h->stream);
+                              beside ? h->tail_stream : h->stream);
             h->launches += 1;
+            if (beside && e == cudaSuccess) {
+                e = cudaEventRecord(h->ev_join, h->tail_stream);
+                if (e == cudaSuccess) e = cudaStreamWaitEvent(h->stream, h->ev_join, 0);
+            }
             if (pipe && e == cudaSuccess) {
                 e = cudaEventRecord(h->ev_done[r], h->stream);
                 if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_done[r], 0);
@@ -946,6 +970,9 @@ int lazyev_destroy(lazyev_t* h) {
         cudaEventDestroy(sp.stop);
     }
     for (cudaEvent_t e : h->free_events) cudaEventDestroy(e);
+    if (h->tail_stream) cudaStreamDestroy(h->tail_stream);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
     if (h->copy_in) cudaStreamDestroy(h->copy_in);
     if (h->copy_out) cudaStreamDestroy(h->copy_out);
     for (int i = 0; i <= kHostChunks; ++i) {
