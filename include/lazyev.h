@@ -14,7 +14,11 @@
  *     that was current at lazyev_bind(); activations are bfloat16 (raw 16-bit
  *     patterns), head_dim = 128 elements per row.
  *   - The caller owns all device memory and the CUDA stream.  The library
- *     allocates no device memory at all; it owns only the host-side handle.
+ *     allocates no device memory at all; it owns only the host-side handle and a
+ *     few internal CUDA streams and events (a low-priority stream for the second
+ *     decode launch of a step, two copy streams for the host-buffer entry point),
+ *     created on first use and destroyed with the handle; their work is always
+ *     joined into the bound stream before a call returns control to it.
  *   - Calls are asynchronous on the bound stream unless stated otherwise.
  *     A handle must not be used from two threads at once.
  *
@@ -27,7 +31,8 @@
  *             in physical page page_table[u][i / 64], row i % 64.
  *   state   : page table, and per unit and slot: TS (int32), MRI (int32),
  *             original position (int32), last probability (float32).
- *   scratch : eviction source lists, staging for the host-buffer entry point.
+ *   scratch : eviction source lists, staging for the host-buffer entry point, score
+ *             staging for lazyev_dump_state, the MRI histogram.
  */
 #ifndef LAZYEV_H
 #define LAZYEV_H
