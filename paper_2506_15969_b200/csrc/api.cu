@@ -260,11 +260,10 @@ struct HostPipe {
 int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPipe* pipe) {
     cudaError_t e = cudaSuccess;
     DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages, h->force_groups};
-    // Launch shape, chosen per number of pages in use and cached.  Every cluster size whose logits fit
-    // gets a relative speed (blocks per unit, discounted for the per-unit exchange between the blocks
-    // of a cluster and for a shallow page ring); the main launch is the size with the least time over
-    // the rounds of the round-robin walk.  A partly filled last round goes to a second launch with
-    // larger clusters when that is faster, so that more SMs share its units.
+    // Launch shape, chosen per number of pages in use and cached.  For every cluster size whose logits
+    // fit, a small time model gives the time of the rounds of the round-robin walk; the main launch is
+    // the size with the least total.  A partly filled last round goes to a second launch with larger
+    // clusters when that is faster, so that more SMs share its units.
     const int np = (n + kPageTokens - 1) / kPageTokens;
     auto cached = h->plan_cache.find(np);
     if (cached == h->plan_cache.end() || cached->second.forced_splits != h->force_splits ||
@@ -273,11 +272,14 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
         best.forced_splits = h->force_splits;
         best.forced_stages = h->force_stages;
         best.forced_groups = h->force_groups;
-        // relative speed of one block by ring depth and by cluster size (measured on B200 at 8 k tokens)
+        // Time model, in units of the time one block needs for one page when it is not limited by HBM
+        // (fitted on B200 at 8 k tokens per unit): a round of `m` units on clusters of s blocks takes
+        //   max(pages per block + kFixedPages, kHbmPageTime * m * np / SMs) / ring weight
+        // -- a fixed cost per unit (merge, pipeline refill), and the HBM floor once many SMs stream; a second
+        // launch costs kSecondLaunchPages on top of its round.
         static const double kRingWeight[7] = {0, 0, 0.70, 0.90, 0.96, 0.99, 1.0};
-        static const double kSplitWeight[9] = {0, 1.0, 0.94, 0.92, 0.90, 0.88, 0.86, 0.84, 0.82};
-        int max_clusters[9] = {0};
-        double speed[9] = {0};                       // units per unit of time done by one cluster of s blocks
+        constexpr double kFixedPages = 8.0, kHbmPageTime = 1.12, kSecondLaunchPages = 10.0;
+        int max_clusters[9] = {0}, stages_of[9] = {0};
         for (int s = 1; s <= 8; ++s) {
             if (h->force_splits == 0 && s > 1 && (np < 2 * s)) continue;       // at least two pages per block
             DecodePlan plan;
@@ -289,26 +291,33 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
                 continue;
             }
             max_clusters[s] = clusters;
-            speed[s] = s * kRingWeight[plan.stages] * kSplitWeight[s];
+            stages_of[s] = plan.stages;
         }
+        auto round_time = [&](int s, int m) {
+            const double own = (double)((np + s - 1) / s) + kFixedPages;
+            const double hbm = kHbmPageTime * (double)m * np / h->num_sms;
+            return (own > hbm ? own : hbm) / kRingWeight[stages_of[s]];
+        };
         double best_time = -1.0;
         for (int s = 1; s <= 8; ++s) {
             if (max_clusters[s] < 1 || (h->force_splits > 0 && s != h->force_splits)) continue;
             const int used = max_clusters[s] < h->units ? max_clusters[s] : h->units;
             const int full = h->units / used, rem = h->units % used;
-            double time = full / speed[s];
+            double time = full * round_time(s, used);
             int ts = 0;
             if (rem > 0) {
-                double tail = 1.0 / speed[s];
+                // the partly filled last round: as it is, or in a second launch with larger clusters
+                double tail = round_time(s, rem);
                 if (full > 0 && h->force_splits == 0)
                     for (int k = s + 1; k <= 8; ++k)
-                        if (max_clusters[k] >= rem && rem * k <= h->num_sms && 1.0 / speed[k] < tail) {
-                            tail = 1.0 / speed[k];
+                        if (max_clusters[k] >= rem && rem * k <= h->num_sms &&
+                            round_time(k, rem) + kSecondLaunchPages < tail) {
+                            tail = round_time(k, rem) + kSecondLaunchPages;
                             ts = k;
                         }
                 time += tail;
             }
-            if (best_time < 0 || time < best_time - 1e-12) {
+            if (best_time < 0 || time < 0.98 * best_time) {      // larger clusters only for a clear gain
                 best_time = time;
                 best.splits = s;
                 best.clusters = used;

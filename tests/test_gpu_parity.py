@@ -36,7 +36,7 @@ def test_attention_and_tracking_without_eviction(splits):
 
 def test_partly_filled_last_round_goes_to_a_second_launch():
     """158 units on 148 SMs: 148 in the main launch, the other 10 in a launch with larger clusters."""
-    cfg = traces.tiny_config(batch=2, layers=79, q_heads=7, kv_heads=1, budget=300, window=32, prefill=280)
+    cfg = traces.tiny_config(batch=2, layers=79, q_heads=7, kv_heads=1, budget=1520, window=32, prefill=1500)
     ls = lockstep(cfg, seed=14, sample_units=[0, 1, 147, 148, 149, 156, 157], pure=False)
     ls.run(40)
     ls.assert_ok()
