@@ -470,69 +470,106 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 }
             }
             named_barrier_sync(1, kConsumers);
-            Xchg* xb = xchg + (it & 1);
-            if (ctid < kMaxGroup * NW) {
-                const int w = ctid >> 3, h = ctid & 7;
-                float mc = -INFINITY;
+            if (!clustered) {
+                // One block owns the unit: every warp finishes 8 / NW heads on its own -- the block's
+                // reference, the per-warp scales, l, the log-sum-exp and the normalised output -- so one
+                // more barrier (for the log-sum-exp) ends the unit.
+                constexpr int kHeadsPerWarp = kMaxGroup / NW;
 #pragma unroll
-                for (int k = 0; k < NW; ++k) mc = fmaxf(mc, wml[k * 16 + h]);
-                const float mw = wml[w * 16 + h];
-                scw[w * kMaxGroup + h] = mw == -INFINITY ? 0.f : fast_exp2(mw - mc);
-                if (w == 0) {
-                    float lc = 0.f;
+                for (int hh = 0; hh < kHeadsPerWarp; ++hh) {
+                    const int h = warp * kHeadsPerWarp + hh;
+                    float mc = -INFINITY;
+#pragma unroll
+                    for (int k = 0; k < NW; ++k) mc = fmaxf(mc, wml[k * 16 + h]);
+                    float sc[NW], lc = 0.f;
 #pragma unroll
                     for (int k = 0; k < NW; ++k) {
                         const float mk = wml[k * 16 + h];
-                        lc += mk == -INFINITY ? 0.f : wml[k * 16 + 8 + h] * fast_exp2(mk - mc);
+                        sc[k] = mk == -INFINITY ? 0.f : fast_exp2(mk - mc);
+                        lc += wml[k * 16 + 8 + h] * sc[k];
                     }
-                    xb->m[h] = mc;
-                    xb->l[h] = lc;
-                }
-            }
-            named_barrier_sync(1, kConsumers);
-            for (int e = ctid; e < kMaxGroup * kHeadDim; e += kConsumers) {
-                const int h = e >> 7, d = e & (kHeadDim - 1);
-                float acc = 0.f;
+                    const float inv = 1.f / lc;
+                    if (lane == 0) lse_s[h] = mc + log2f(lc);
+                    if (h < G) {
 #pragma unroll
-                for (int k = 0; k < NW; ++k) acc += slots[k * (kMaxGroup * kXchgRow) + h * kXchgRow + d] * scw[k * kMaxGroup + h];
-                xb->o[h][d] = acc;
-            }
-            if (clustered) {
-                cluster_arrive();
-                cluster_wait();
-            } else {
+                        for (int k4 = 0; k4 < kHeadDim / 32; ++k4) {
+                            const int d = lane + 32 * k4;
+                            float acc = 0.f;
+#pragma unroll
+                            for (int k = 0; k < NW; ++k) acc += slots[k * (kMaxGroup * kXchgRow) + h * kXchgRow + d] * sc[k];
+                            p.out[((size_t)u * G + h) * kHeadDim + d] = __float2bfloat16_rn(acc * inv);
+                        }
+                    }
+                }
                 named_barrier_sync(1, kConsumers);
-            }
-
-            // ---- merge the blocks of the cluster: exact log-sum-exp per head -----
-            if (ctid < kMaxGroup) {
-                float M = -INFINITY, L = 0.f;
-                for (int r = 0; r < S; ++r) M = fmaxf(M, ld_rank_f32(&xb->m[ctid], r, clustered));
-                for (int r = 0; r < S; ++r) {
-                    const float mr = ld_rank_f32(&xb->m[ctid], r, clustered);
-                    L += mr == -INFINITY ? 0.f : ld_rank_f32(&xb->l[ctid], r, clustered) * exp2f(mr - M);
+                lse0 = lse_s[h0];
+                lse1 = lse_s[h1];
+                u_prev = u;
+            } else {
+                Xchg* xb = xchg + (it & 1);
+                if (ctid < kMaxGroup * NW) {
+                    const int w = ctid >> 3, h = ctid & 7;
+                    float mc = -INFINITY;
+#pragma unroll
+                    for (int k = 0; k < NW; ++k) mc = fmaxf(mc, wml[k * 16 + h]);
+                    const float mw = wml[w * 16 + h];
+                    scw[w * kMaxGroup + h] = mw == -INFINITY ? 0.f : fast_exp2(mw - mc);
+                    if (w == 0) {
+                        float lc = 0.f;
+#pragma unroll
+                        for (int k = 0; k < NW; ++k) {
+                            const float mk = wml[k * 16 + h];
+                            lc += mk == -INFINITY ? 0.f : wml[k * 16 + 8 + h] * fast_exp2(mk - mc);
+                        }
+                        xb->m[h] = mc;
+                        xb->l[h] = lc;
+                    }
                 }
-                lse_s[ctid] = M + log2f(L);
-                for (int r = 0; r < S; ++r) {
-                    const float mr = ld_rank_f32(&xb->m[ctid], r, clustered);
-                    sc_s[r * kMaxGroup + ctid] = mr == -INFINITY ? 0.f : exp2f(mr - M) / L;
-                }
-            }
-            named_barrier_sync(1, kConsumers);
-            lse0 = lse_s[h0];
-            lse1 = lse_s[h1];
-            u_prev = u;
-
-            // out[g][d]: each block of the cluster finishes a slice of the head dimension
-            {
-                const int d_lo = kHeadDim * (int)rank / S, d_hi = kHeadDim * ((int)rank + 1) / S;
-                const int dper = d_hi - d_lo;
-                for (int e = ctid; e < G * dper; e += kConsumers) {
-                    const int gg = e / dper, d = d_lo + e % dper;
+                named_barrier_sync(1, kConsumers);
+                for (int e = ctid; e < kMaxGroup * kHeadDim; e += kConsumers) {
+                    const int h = e >> 7, d = e & (kHeadDim - 1);
                     float acc = 0.f;
-                    for (int r = 0; r < S; ++r)
-                        acc += ld_rank_f32(&xb->o[gg][d], r, clustered) * sc_s[r * kMaxGroup + gg];
-                    p.out[((size_t)u * G + gg) * kHeadDim + d] = __float2bfloat16_rn(acc);
+#pragma unroll
+                    for (int k = 0; k < NW; ++k) acc += slots[k * (kMaxGroup * kXchgRow) + h * kXchgRow + d] * scw[k * kMaxGroup + h];
+                    xb->o[h][d] = acc;
+                }
+                if (clustered) {
+                    cluster_arrive();
+                    cluster_wait();
+                } else {
+                    named_barrier_sync(1, kConsumers);
+                }
+
+                // ---- merge the blocks of the cluster: exact log-sum-exp per head -----
+                if (ctid < kMaxGroup) {
+                    float M = -INFINITY, L = 0.f;
+                    for (int r = 0; r < S; ++r) M = fmaxf(M, ld_rank_f32(&xb->m[ctid], r, clustered));
+                    for (int r = 0; r < S; ++r) {
+                        const float mr = ld_rank_f32(&xb->m[ctid], r, clustered);
+                        L += mr == -INFINITY ? 0.f : ld_rank_f32(&xb->l[ctid], r, clustered) * exp2f(mr - M);
+                    }
+                    lse_s[ctid] = M + log2f(L);
+                    for (int r = 0; r < S; ++r) {
+                        const float mr = ld_rank_f32(&xb->m[ctid], r, clustered);
+                        sc_s[r * kMaxGroup + ctid] = mr == -INFINITY ? 0.f : exp2f(mr - M) / L;
+                    }
+                }
+                named_barrier_sync(1, kConsumers);
+                lse0 = lse_s[h0];
+                lse1 = lse_s[h1];
+                u_prev = u;
+
+                // out[g][d]: each block of the cluster finishes a slice of the head dimension
+                {
+                    const int d_lo = kHeadDim * (int)rank / S, d_hi = kHeadDim * ((int)rank + 1) / S;
+                    const int dper = d_hi - d_lo;
+                    for (int e = ctid; e < G * dper; e += kConsumers) {
+                        const int gg = e / dper, d = d_lo + e % dper;
+                        float acc = 0.f;
+                        for (int r = 0; r < S; ++r)
+                            acc += ld_rank_f32(&xb->o[gg][d], r, clustered) * sc_s[r * kMaxGroup + gg];
+                        p.out[((size_t)u * G + gg) * kHeadDim + d] = __float2bfloat16_rn(acc);
+                    }
                 }
             }
 #pragma unroll
