@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # 592-unit case of the same launch shape; traffic grows in proportion to units x tokens, so a full
 # launch is scaled by its algorithmic bytes.  Valid only for the kernel sources it was taken on.
 NCU_DECODE_CAPTURE = {
-    "traffic_per_algorithmic_byte": 1.0076,
-    "sha256": {"decode.cu": "bda937e979593d4cd5a8b5d0b94513609ccbc60fb249bc06cf23f52216c32184",
+    "traffic_per_algorithmic_byte": 1.0075,
+    "sha256": {"decode.cu": "a4ecc7346b7141d70069dd3e73dafa326a2d20008d509c194be4842d22ef22ba",
                "common.cuh": "e145966ccf290b94a07f9b5374ce552520833824b6b9440fc6aa85adf416adac"},
 }
 
