@@ -35,10 +35,10 @@ if ROOT not in sys.path:
 
 METRIC = "decode tokens/sec (all layers, batch B) and fraction of B200 HBM roofline"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM traffic of the decode kernel from the ncu capture summarised in
-# profiles/decode_kernel_cfg4_small_ncu.md: (dram read + write bytes) / algorithmic bytes on a
-# 592-unit case of the same launch shape; traffic grows in proportion to units x tokens, so a full
-# launch is scaled by its algorithmic bytes.  Valid only for the kernel sources it was taken on.
+# DRAM traffic of the decode kernel from the committed ncu capture of a 592-unit case of the same
+# launch shape: (dram read + write bytes) / algorithmic bytes; traffic grows in proportion to
+# units x tokens, so a full launch is scaled by its algorithmic bytes.  Valid only for the kernel
+# sources it was taken on.
 NCU_DECODE_CAPTURE = {
     "traffic_per_algorithmic_byte": 1.0075,
     "sha256": {"decode.cu": "a4ecc7346b7141d70069dd3e73dafa326a2d20008d509c194be4842d22ef22ba",
@@ -68,20 +68,25 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4)
     ap.add_argument("--seed", type=int, default=0)
-    ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch (profiling on small cases)")
-    ap.add_argument("--layers", type=int, default=0, help="override the configuration's layer count (profiling on small cases)")
-    ap.add_argument("--start-step", type=int, default=-1,
-                    help="decode steps replayed untimed before the timed region (-1: up to the first eviction)")
-    ap.add_argument("--fast-start", action="store_true",
-                    help="prefill a prompt as long as the budget instead of replaying the trace up to it")
-    ap.add_argument("--splits", type=int, default=0)
-    ap.add_argument("--stages", type=int, default=0)
-    ap.add_argument("--groups", type=int, default=0)
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--no-profile", action="store_true")
+    ap.add_argument("--alpha", type=float, default=0.0,
+                    help="importance threshold (default: the configuration's 8 / (budget + window); the paper's own "
+                         "1e-4 .. 5e-4 give the dense-activation regime)")
     ap.add_argument("--cpu-units", type=int, default=0)
     ap.add_argument("--cpu-steps", type=int, default=0)
+    pc = ap.add_argument_group("profile-case", "shape a small case of the same kernels for an ncu capture, or skip legs "
+                                               "of the run; none of these is used for a headline number")
+    pc.add_argument("--batch", type=int, default=0, help="override the configuration's batch")
+    pc.add_argument("--layers", type=int, default=0, help="override the configuration's layer count")
+    pc.add_argument("--start-step", type=int, default=-1,
+                    help="decode steps replayed untimed before the timed region (-1: up to the first eviction)")
+    pc.add_argument("--fast-start", action="store_true",
+                    help="prefill a prompt as long as the budget instead of replaying the trace up to it")
+    pc.add_argument("--splits", type=int, default=0)
+    pc.add_argument("--stages", type=int, default=0)
+    pc.add_argument("--groups", type=int, default=0)
+    pc.add_argument("--no-e2e", action="store_true")
+    pc.add_argument("--no-cpu", action="store_true")
+    pc.add_argument("--no-profile", action="store_true")
     return ap.parse_args()
 
 
@@ -95,6 +100,8 @@ def pick_config(args):
     if args.fast_start:
         cfg = dataclasses.replace(cfg, prefill=cfg.budget_at(0) if cfg.budget_frac_tenths else cfg.budget,
                                   name=cfg.name + "-faststart")
+    if args.alpha > 0:
+        cfg = dataclasses.replace(cfg, alpha=args.alpha, name=f"{cfg.name}-alpha{args.alpha:g}")
     return cfg
 
 
@@ -153,7 +160,7 @@ class ClockSampler(threading.Thread):
                 for bit, name in names.items():
                     if mask & bit:
                         self.reasons.add(name)
-                time.sleep(0.05)
+                time.sleep(0.01)
         except Exception as e:  # pragma: no cover
             self.reasons.add(f"nvml_unavailable:{type(e).__name__}")
 
@@ -267,13 +274,17 @@ def run_ours(args):
 
     t = 0
 
-    def run_chunk(cnt, host=False, timed=False):
-        """Generate `cnt` steps of inputs (untimed), then run them; returns device ms (or wall ms for host)."""
+    last_host = {}
+
+    def run_chunk(cnt, host=None):
+        """Generate `cnt` steps of inputs (untimed), then run them; returns device ms (wall ms for the host
+        entry points).  host: None = resident inputs, "sync" = lazyev_decode_step_host, "async" =
+        lazyev_decode_step_host_async with one step in flight behind the one being queued."""
         nonlocal t
         q, kn, vn = gen.steps(cnt)
         if host:
             qh, kh, vh = q.cpu().pin_memory(), kn.cpu().pin_memory(), vn.cpu().pin_memory()
-            oh = torch.empty(out.shape, dtype=torch.bfloat16).pin_memory()
+            oh = [torch.empty(out.shape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         w0 = time.perf_counter()
@@ -282,12 +293,19 @@ def run_ours(args):
             t += 1
             if cfg.budget_frac_tenths and t % cfg.window == 0:
                 eng.set_budget(cfg.budget_at(t))
-            if host:
-                eng.decode_step_host(qh[s], kh[s], vh[s], oh)
+            if host == "sync":
+                eng.decode_step_host(qh[s], kh[s], vh[s], oh[s & 1])
+            elif host == "async":
+                eng.decode_step_host_async(qh[s], kh[s], vh[s], oh[s & 1])
+                eng.host_wait(1)             # the step before this one is complete: its output is on the host
             else:
                 eng.decode_step(q[s], kn[s], vn[s], out)
+        if host == "async":
+            eng.host_wait(0)
         e1.record(stream)
         torch.cuda.synchronize()
+        if host:
+            last_host.update(q=q[cnt - 1], k=kn[cnt - 1], v=vn[cnt - 1], out=oh[(cnt - 1) & 1])
         return (time.perf_counter() - w0) * 1e3 if host else e0.elapsed_time(e1)
 
     def run_steps(count, **kw):
@@ -313,8 +331,7 @@ def run_ours(args):
     sampler.start()
     ms = run_steps(args.steps)
     barrier()
-    sampler.stop_flag = True
-    sampler.join(timeout=2)
+    timed_samples = len(sampler.samples)
     launches = eng.info().launches - launches0
     evictions_timed = sum(1 for x in range(t_first, t + 1) if x % cfg.window == 0)
     ms = replicas.max_over_ranks(ms, dist, "cuda")
@@ -322,7 +339,7 @@ def run_ours(args):
     value = replicas.job_tokens_per_second(cfg.batch, args.steps, world, ms)
 
     # ---- per-kernel roofline: one observation window with events around each kernel ----
-    roofline, kernels = None, None
+    roofline, kernels, value_amortised = None, None, None
     if not args.no_profile:
         eng.set_profiling(True)
         eng.get_profile(reset=True)
@@ -330,39 +347,88 @@ def run_ours(args):
         pr = eng.get_profile(reset=True)
         eng.set_profiling(False)
         peak, peak_kind = measured_peak()
-        dec_gbs = pr.decode_bytes / (pr.decode_ms * 1e-3) / 1e9
+        # Tokens at or above the threshold cost the epilogue a TS read, an MRI read-modify-write and a TS
+        # write on top of the 512 + 4 bytes every token costs: up to 16 bytes each.  Their share is read off
+        # the state of a few units after the last profiled step (TS = t marks a token activated by it).
+        su = list(range(0, cfg.units, max(1, cfg.units // 8)))[:8]
+        act = sum(float((eng.dump_state(u, 1)["ts"][0] == t).mean()) for u in su) / len(su)
+        launches_p = max(pr.decode_launches, 1)
+        dec_bytes = pr.decode_bytes + 16.0 * act * (pr.decode_bytes / 516.0)
+        dec_gbs = dec_bytes / (pr.decode_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": "decode_kernel (attention + probabilities + TS/MRI update)",
                     "achieved": round(dec_gbs, 1), "peak": peak, "unit": "GB/s", "frac": round(dec_gbs / peak, 4),
                     "peak_kind": peak_kind, "frac_of_8TBps_nominal": round(dec_gbs / 8000.0, 4),
-                    "traffic": ncu_traffic(pr.decode_bytes / max(pr.decode_launches, 1)),
+                    "traffic": ncu_traffic(pr.decode_bytes / launches_p),
                     "traffic_source": "ncu dram__bytes_read+write on a 592-unit case of the same launch shape, "
                                       "scaled by algorithmic bytes (null if the kernel changed since)",
-                    "ms_per_launch": round(pr.decode_ms / max(pr.decode_launches, 1), 4),
-                    "bytes_per_launch": pr.decode_bytes / max(pr.decode_launches, 1)}
+                    "ms_per_launch": round(pr.decode_ms / launches_p, 4),
+                    "bytes_per_launch": dec_bytes / launches_p,
+                    "activated_share_of_tokens": round(act, 4),
+                    "achieved_without_state_bytes": round(pr.decode_bytes / (pr.decode_ms * 1e-3) / 1e9, 1)}
         kernels = {"append_ms_per_launch": round(pr.append_ms / max(pr.append_launches, 1), 4)}
         if pr.compact_launches:
             cgbs = pr.compact_bytes / (pr.compact_ms * 1e-3) / 1e9
+            egbs = (pr.compact_bytes + pr.select_bytes) / ((pr.compact_ms + pr.select_ms) * 1e-3) / 1e9
             kernels.update({
                 "compact_ms_per_event": round(pr.compact_ms / pr.compact_launches, 4),
                 "compact_GBps": round(cgbs, 1), "compact_frac_of_measured": round(cgbs / peak, 4),
                 "compact_frac_of_8TBps_nominal": round(cgbs / 8000.0, 4),
+                "compact_rows_per_unit": round(pr.compact_rows / pr.compact_launches / cfg.units, 1),
                 "select_ms_per_event": round(pr.select_ms / pr.select_launches, 4),
-                "select_GBps": round(pr.select_bytes / (pr.select_ms * 1e-3) / 1e9, 1)})
+                "select_GBps": round(pr.select_bytes / (pr.select_ms * 1e-3) / 1e9, 1),
+                "eviction_event_ms": round((pr.compact_ms + pr.select_ms) / pr.compact_launches, 4),
+                "eviction_event_GBps": round(egbs, 1), "eviction_event_frac_of_measured": round(egbs / peak, 4),
+                "eviction_event_frac_of_8TBps_nominal": round(egbs / 8000.0, 4)})
+            cnt = eng.counters()
+            kernels["select_route_units"] = {"radix": cnt.select_radix_units, "zero_cut": cnt.select_zero_cut_units}
+            if evictions_timed == 0:
+                # the timed steps held no decision step: the same figure with one eviction per window spread over it
+                per_step = ms / args.steps + (pr.compact_ms + pr.select_ms) / pr.compact_launches / cfg.window
+                value_amortised = cfg.batch * world / (per_step * 1e-3)
 
     # ---- end to end: the same steps from pinned host buffers through the C ABI ----------
     e2e = None
     if not args.no_e2e:
-        run_steps(3, host=True)
+        run_steps(3, host="async")
         e2e_steps = min(args.steps, cfg.window)
         barrier()
-        wall_ms = run_steps(e2e_steps, host=True)
+        wall_ms = run_steps(e2e_steps, host="async")
         barrier()
         wall_ms = replicas.max_over_ranks(wall_ms, dist, "cuda")
+        sync_steps = min(e2e_steps, 32)
+        sync_ms = replicas.max_over_ranks(run_steps(sync_steps, host="sync"), dist, "cuda")
         qbytes = L * Bt * cfg.q_heads * cfg.head_dim * 2
         kbytes = L * Bt * cfg.kv_heads * cfg.head_dim * 2
         e2e = {"value": replicas.job_tokens_per_second(cfg.batch, e2e_steps, world, wall_ms), "unit": "tokens/s",
                "h2d_bytes_per_step": qbytes + 2 * kbytes, "d2h_bytes_per_step": qbytes, "steps": e2e_steps,
-               "ms_per_step": wall_ms / e2e_steps}
+               "ms_per_step": wall_ms / e2e_steps,
+               "call": "lazyev_decode_step_host_async + lazyev_host_wait(1) per step (uploads of step t+1 and the "
+                       "download of step t-1 run beside the kernels of step t)",
+               "sync_call": {"call": "lazyev_decode_step_host (returns with the output on the host)",
+                             "value": replicas.job_tokens_per_second(cfg.batch, sync_steps, world, sync_ms),
+                             "ms_per_step": sync_ms / sync_steps, "steps": sync_steps}}
+        # The host-buffer entry points against the resident one on the same state: a fork of the cache takes the
+        # next step with resident inputs while this handle takes it through each host call; outputs must be equal.
+        if world == 1:
+            twin = binding.Engine(cfg.layers, cfg.q_heads, cfg.kv_heads, cfg.head_dim, cfg.budget, cfg.window,
+                                  cfg.threshold, batch=cfg.batch, n_recent=cfg.n_recent, n_initial=cfg.n_initial,
+                                  max_prefill=cfg.prefill)
+            out_twin = torch.empty_like(out)
+            checks = {}
+            for kind in ("async", "sync"):
+                twin.reset()
+                twin.copy_state_from(eng)
+                run_steps(1, host=kind)
+                twin.decode_step(last_host["q"], last_host["k"], last_host["v"], out_twin)
+                twin.synchronize()
+                checks[kind] = bool(torch.equal(out_twin.cpu(), last_host["out"]))
+            e2e["outputs_equal_resident_step"] = checks
+            if not all(checks.values()):
+                raise SystemExit(f"host-buffer step differs from the resident step on the same state: {checks}")
+            twin.close()
+            del twin, out_twin
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
     eng.synchronize()
 
     # ---- the oracle on the host cores, bounded sample (rank 0, one GPU only) ----------------
@@ -380,6 +446,7 @@ def run_ours(args):
         line = {
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "value_amortised": value_amortised,
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"{cfg.name}: steps {t_first}..{t_first + args.steps - 1} of the seeded trace "
                                    f"(cache {inf.budget_now}+1..{inf.budget_now}+{cfg.window} tokens per unit, "
@@ -392,7 +459,9 @@ def run_ours(args):
                                          "tail_units": inf.tail_units, "tail_splits": inf.tail_splits,
                                          "smem_bytes": inf.smem_bytes},
                        "multi_gpu": "independent replicas of the batch per GPU, no collective"},
-            "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": dict(sampler.summary(), samples_in_timed_region=timed_samples,
+                           window="timed steps, per-kernel pass and host-buffer pass"),
+            "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu,
         }
         print(json.dumps(line))

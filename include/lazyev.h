@@ -164,7 +164,13 @@ int lazyev_prefill_observed(lazyev_t* h, const void* q, const void* k, const voi
  * q, out: [layers, batch, q_heads, head_dim]; k_new, v_new: [layers, batch,
  * kv_heads, head_dim]; all device pointers, bf16.
  * Errors: ESTATE (no prefill), ECAPACITY (cache full: eviction was disabled
- * and never called), ECUDA.  Failures that kernels detect (a bounded wait that
+ * and never called), EINVAL (automatic eviction is on and this step's eviction
+ * would run over more candidates than lazyev_evict() supports), ECUDA.  All of
+ * these are found before anything is queued: the step did not happen and may
+ * be retried after the cause is removed.  The one exception is ECUDA from a
+ * kernel launch: the launches of a step are queued one after the other, so a
+ * launch failure leaves the handle in an undefined state (destroy it).
+ * Failures that kernels detect (a bounded wait that
  * gave up, an index out of range) are recorded in a device status word and
  * reported by lazyev_synchronize() and lazyev_dump_state() as EDEVICE.
  */
@@ -175,6 +181,36 @@ int lazyev_decode_step(lazyev_t* h, const void* q, const void* k_new, const void
  * synchronises.  Queries and outputs move in unit ranges on two internal copy streams
  * (created at the first call) while the decode launches of the other ranges run. */
 int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out);
+
+/*
+ * The same step with host buffers, without waiting for it: the call queues the uploads, the
+ * step and the download of `out` and returns.  Two steps may be in flight at once; the inputs
+ * of step t + 1 are uploaded while the kernels of step t run, and the output of step t comes
+ * back while step t + 1 runs, so a caller that has the next inputs ready (another micro-batch,
+ * a replayed trace) pays for the copies only where they exceed the kernel time.  A call that
+ * finds two steps in flight first waits for the older one.  The host buffers of a step belong
+ * to the library until lazyev_host_wait() says the step is complete: q, k_new and v_new must
+ * not change and `out` must not be read before that.  Errors as for lazyev_decode_step().
+ * (The paper decodes one sequence batch synchronously; this is a serving convenience.)
+ */
+int lazyev_decode_step_host_async(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out);
+/* Blocks until at most `in_flight_allowed` (0 or 1) of the steps queued with
+ * lazyev_decode_step_host_async() are incomplete: with 1, everything but the newest step is
+ * finished and its `out` may be read.  Errors: EINVAL, ECUDA. */
+int lazyev_host_wait(lazyev_t* h, int in_flight_allowed);
+
+/*
+ * Fork: make `dst` hold an exact copy of the sequences cached in `src` (pool pages, page table,
+ * TS, MRI, positions, probabilities, counters, t, n, budget_now), device to device, ordered
+ * after everything queued on src's stream and asynchronous on dst's stream (src's stream in
+ * turn waits for the copy before it runs anything queued later).  Both handles must
+ * be bound on the same device with the same shape, budget, window and protection settings;
+ * dst must hold no cache yet (fresh or reset).  Afterwards the two handles decode
+ * independently and, given the same inputs, identically.  (No counterpart in the paper; used to
+ * branch a generation and to check one entry point against another on the same state.)
+ * Errors: EINVAL (different configurations), ESTATE, ECUDA.
+ */
+int lazyev_copy_state(lazyev_t* dst, lazyev_t* src);
 
 /*
  * Lagged eviction (Section 4 "MRI-Centric Eviction", Eq. 2, Eq. evic): if t is
@@ -191,8 +227,8 @@ int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const
 int lazyev_evict(lazyev_t* h, int* evicted);
 
 /*
- * lazyev_evict() for callers that have no scratch region to spare.  (The paper has no
- * counterpart; this is a deployment convenience.)
+ * lazyev_evict() with its work lists inside the library.  (The paper has no counterpart; this
+ * is a deployment convenience.)
  *
  * Who needs it: code that runs where device allocation is off the table -- a plug-in inside a
  * serving process that hands out one fixed arena at start-up and treats any later cudaMalloc
@@ -202,10 +238,13 @@ int lazyev_evict(lazyev_t* h, int* evicted);
  * outputs), but wants the eviction's work lists to come from somewhere else.
  *
  * This entry point does exactly what lazyev_evict() does -- same trigger test, same kernels,
- * same results bit for bit -- but keeps the source lists and first-moved indices in an array
- * that is compiled into the library (4 MiB + 16 KiB of device memory on every GPU that loads
- * the library, held until the process exits) instead of the scratch region given to
- * lazyev_bind().  It calls no allocator of any kind.
+ * same results bit for bit, same profiling records -- but keeps the source lists and
+ * first-moved indices (the part of the scratch region that grows with units * budget) in an
+ * array that is compiled into the library (4 MiB + 16 KiB of device memory on every GPU that
+ * loads the library, held until the process exits).  It calls no device allocator of any kind.
+ * lazyev_bind() still wants a scratch region of the size lazyev_query_sizes() reports (the
+ * staging buffers and the 256 KiB table of H2 terms live there); a caller that only ever uses
+ * this entry point may leave its first units * budget * 4 bytes untouched by anything else.
  *
  * Limits: units <= 4096 and units * budget_now <= 1,048,576 (2^20) source indices; a larger
  * handle gets LAZYEV_ECAPACITY and a message naming both numbers, before anything runs.
@@ -236,9 +275,25 @@ typedef struct lazyev_info {
     int smem_bytes;      /* dynamic shared memory of the last decode launch  */
     long long launches;  /* kernels launched by this handle so far           */
     long long evictions; /* eviction events so far                           */
+    int host_ranges;     /* unit ranges (decode launches) the last lazyev_decode_step_host call was split into */
 } lazyev_info_t;
 
 int lazyev_get_info(const lazyev_t* h, lazyev_info_t* out);
+
+/*
+ * Event counters kept on the device (tests and diagnostics); synchronises the stream.  They
+ * count since lazyev_bind() or the last lazyev_reset().  The selection of an eviction
+ * (Appendix A, Eq. (evic)) has two routes per unit: when no more than k candidates have a
+ * non-zero score the k-th score is 0 and only the tie rule is left (select_zero_cut_units);
+ * otherwise a radix select over the score bits finds the k-th score (select_radix_units).
+ */
+typedef struct lazyev_counters {
+    int device_status;            /* the kernels' status word (0 = healthy)      */
+    int select_radix_units;
+    int select_zero_cut_units;
+} lazyev_counters_t;
+
+int lazyev_get_counters(lazyev_t* h, lazyev_counters_t* out);
 
 /*
  * Snapshot for tests and checkpoints; synchronises the stream.  The caller

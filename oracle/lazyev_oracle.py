@@ -195,12 +195,45 @@ class OracleUnit:
         self.t = 0
         self.P = 0
         self.pos = np.zeros(0, dtype=np.int64)
-        self.K = np.zeros((0, self.D))
-        self.V = np.zeros((0, self.D))
+        self._set_rows(np.zeros((0, self.D)), np.zeros((0, self.D)))
         self.TS = np.zeros(0, dtype=np.int64)
         self.MRI = np.zeros(0, dtype=np.int64)
         self.last_pbar = np.zeros(0)
         self.last_evict = None             # dict describing the latest eviction
+
+    # -- storage of the cached rows ------------------------------------------------
+    # K and V are the first n rows of two buffers that grow by doubling, so that appending one
+    # token per step does not copy the whole cache (storage only; no arithmetic lives here).
+    def _set_rows(self, K, V) -> None:
+        self._K = np.array(K, dtype=np.float64)
+        self._V = np.array(V, dtype=np.float64)
+        self._rows = self._K.shape[0]
+
+    def _append_row(self, k_new, v_new) -> None:
+        if self._rows == self._K.shape[0]:
+            grow = max(64, self._rows)
+            self._K = np.vstack([self._K, np.zeros((grow, self.D))])
+            self._V = np.vstack([self._V, np.zeros((grow, self.D))])
+        self._K[self._rows] = np.asarray(k_new, dtype=np.float64)
+        self._V[self._rows] = np.asarray(v_new, dtype=np.float64)
+        self._rows += 1
+
+    @property
+    def K(self) -> np.ndarray:
+        return self._K[: self._rows]
+
+    @K.setter
+    def K(self, rows) -> None:
+        self._K = np.array(rows, dtype=np.float64)
+        self._rows = self._K.shape[0]
+
+    @property
+    def V(self) -> np.ndarray:
+        return self._V[: self._rows]
+
+    @V.setter
+    def V(self, rows) -> None:
+        self._V = np.array(rows, dtype=np.float64)
 
     # -- set-up ---------------------------------------------------------------
     @property
@@ -219,7 +252,7 @@ class OracleUnit:
         V = np.asarray(V, dtype=np.float64)
         self.P = K.shape[0]
         self.pos = np.arange(self.P, dtype=np.int64)
-        self.K, self.V = K.copy(), V.copy()
+        self._set_rows(K, V)
         self.TS = np.zeros(self.P, dtype=np.int64)
         self.MRI = np.zeros(self.P, dtype=np.int64)
         self.t = 0
@@ -236,7 +269,7 @@ class OracleUnit:
         P = K.shape[0]
         self.P = P
         self.pos = np.zeros(0, dtype=np.int64)
-        self.K, self.V = np.zeros((0, self.D)), np.zeros((0, self.D))
+        self._set_rows(np.zeros((0, self.D)), np.zeros((0, self.D)))
         self.TS, self.MRI = np.zeros(0, dtype=np.int64), np.zeros(0, dtype=np.int64)
         self.t = -P                       # attend() advances t before it appends: row j runs at j - (P - 1)
         outs = np.zeros((P, self.G, self.D))
@@ -250,17 +283,20 @@ class OracleUnit:
         return outs
 
     # -- one decode step --------------------------------------------------------
+    def append(self, k_new, v_new) -> None:
+        """t += 1 and the new token joins the cache with TS = t, MRI = 0 (Section 4)."""
+        self.t += 1
+        self.pos = np.append(self.pos, self.P + self.t - 1)
+        self._append_row(k_new, v_new)
+        self.TS = np.append(self.TS, self.t)       # a new token starts at TS = t
+        self.MRI = np.append(self.MRI, 0)          # and MRI = 0 (Section 4)
+
     def attend(self, q, k_new, v_new):
         """t += 1, append the new token, evaluate Eq. (attn).
 
         Returns (out [G, D], pbar [n]) with pbar[i] the group-mean probability.
         """
-        self.t += 1
-        self.pos = np.append(self.pos, self.P + self.t - 1)
-        self.K = np.vstack([self.K, np.asarray(k_new, dtype=np.float64)[None, :]])
-        self.V = np.vstack([self.V, np.asarray(v_new, dtype=np.float64)[None, :]])
-        self.TS = np.append(self.TS, self.t)       # a new token starts at TS = t
-        self.MRI = np.append(self.MRI, 0)          # and MRI = 0 (Section 4)
+        self.append(k_new, v_new)
         out, p = attention(q, self.K, self.V)
         pbar = p.mean(axis=0)
         self.last_pbar = pbar
@@ -314,7 +350,8 @@ class OracleUnit:
 
     def apply_keep(self, kept) -> None:
         kept = np.asarray(kept, dtype=np.int64)
-        self.pos, self.K, self.V = self.pos[kept], self.K[kept], self.V[kept]
+        self._set_rows(self.K[kept], self.V[kept])
+        self.pos = self.pos[kept]
         self.TS, self.MRI = self.TS[kept], self.MRI[kept]
 
     def evict_if_due(self):

@@ -23,7 +23,12 @@ class Info(C.Structure):
     _fields_ = [(n, C.c_int) for n in (
         "layers", "batch", "q_heads", "kv_heads", "head_dim", "units", "budget", "budget_now", "window",
         "n_recent", "n_initial", "capacity", "pages_per_unit", "t", "n", "prefill", "splits", "stages",
-        "groups", "tail_units", "tail_splits", "grid", "smem_bytes")] + [("launches", C.c_longlong), ("evictions", C.c_longlong)]
+        "groups", "tail_units", "tail_splits", "grid", "smem_bytes")] + [("launches", C.c_longlong), ("evictions", C.c_longlong),
+                                                                           ("host_ranges", C.c_int)]
+
+
+class Counters(C.Structure):
+    _fields_ = [("device_status", C.c_int), ("select_radix_units", C.c_int), ("select_zero_cut_units", C.c_int)]
 
 
 class Profile(C.Structure):
@@ -59,9 +64,13 @@ _PROTOS = {
     "lazyev_prefill_observed": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p],
     "lazyev_decode_step": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_decode_step_host": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
+    "lazyev_decode_step_host_async": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
+    "lazyev_host_wait": [C.c_void_p, C.c_int],
+    "lazyev_copy_state": [C.c_void_p, C.c_void_p],
     "lazyev_evict": [C.c_void_p, C.POINTER(C.c_int)],
     "lazyev_evict_static": [C.c_void_p, C.POINTER(C.c_int)],
     "lazyev_get_info": [C.c_void_p, C.POINTER(Info)],
+    "lazyev_get_counters": [C.c_void_p, C.POINTER(Counters)],
     "lazyev_dump_state": [C.c_void_p, C.POINTER(Dump)],
     "lazyev_load_state": [C.c_void_p, C.POINTER(Dump), C.c_int],
     "lazyev_mri_histogram": [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int],
@@ -189,6 +198,16 @@ class Engine:
     def decode_step_host(self, q, k_new, v_new, out) -> None:
         self._check(lib().lazyev_decode_step_host(self._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out)))
 
+    def decode_step_host_async(self, q, k_new, v_new, out) -> None:
+        self._check(lib().lazyev_decode_step_host_async(self._h, _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out)))
+
+    def host_wait(self, in_flight_allowed: int = 0) -> None:
+        self._check(lib().lazyev_host_wait(self._h, in_flight_allowed))
+
+    def copy_state_from(self, src: "Engine") -> None:
+        """lazyev_copy_state(self, src): this handle becomes a copy of src's cached sequences."""
+        self._check(lib().lazyev_copy_state(self._h, src._h))
+
     def evict(self) -> int:
         n = C.c_int()
         self._check(lib().lazyev_evict(self._h, C.byref(n)))
@@ -236,6 +255,11 @@ class Engine:
     def get_profile(self, reset: bool = False) -> Profile:
         out = Profile()
         self._check(lib().lazyev_get_profile(self._h, C.byref(out), int(reset)))
+        return out
+
+    def counters(self) -> Counters:
+        out = Counters()
+        self._check(lib().lazyev_get_counters(self._h, C.byref(out)))
         return out
 
     def info(self) -> Info:

@@ -6,6 +6,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <map>
 #include <utility>
 #include <vector>
@@ -32,18 +33,28 @@ struct lazyev {
     StateView st = {};
     int32_t* src = nullptr;
     int32_t* first_moved = nullptr;
-    uint8_t* stage_q = nullptr;
-    uint8_t* stage_k = nullptr;
-    uint8_t* stage_v = nullptr;
-    uint8_t* stage_out = nullptr;
+    // staging of the host-buffer entry points: two slots, so that the copies of one step run beside
+    // the kernels of the step before it
+    uint8_t* stage_q[2] = {nullptr, nullptr};
+    uint8_t* stage_k[2] = {nullptr, nullptr};
+    uint8_t* stage_v[2] = {nullptr, nullptr};
+    uint8_t* stage_out[2] = {nullptr, nullptr};
     double* stage_score = nullptr;
     unsigned long long* stage_hist = nullptr;
+    double* h2_table = nullptr;            // H2 term per MRI value (scratch), valid for h2_table_mode
+    int h2_table_mode = -1;
     // host-buffer entry point: copy streams and events, created at its first call
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     // second launch of a step (the partly filled last round) runs beside the end of the main launch
     cudaStream_t tail_stream = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     cudaEvent_t ev_in[kHostChunks + 1] = {}, ev_done[kHostChunks + 1] = {}, ev_ready = nullptr;
+    // asynchronous host-buffer steps: completion event per staging slot, steps queued so far, and
+    // whether the slot's last step may still be in flight
+    cudaEvent_t ev_step_done[2] = {nullptr, nullptr};
+    long long host_seq = 0;
+    bool slot_busy[2] = {false, false};
+    int last_host_ranges = 0;
     // progress
     int t = 0, n = 0, prefill = 0;
     long long launches = 0, evictions = 0;
@@ -98,7 +109,7 @@ void derive(lazyev_t* h) {
 struct Sizes {
     size_t kv, state, scratch;
     size_t off_ts, off_mri, off_pos, off_pbar, off_status;                          // inside state
-    size_t off_first, off_q, off_k, off_v, off_out, off_score, off_hist;            // inside scratch
+    size_t off_first, off_q, off_k, off_v, off_out, off_score, off_hist, off_h2;    // inside scratch
 };
 
 Sizes sizes_of(const lazyev_t* h) {
@@ -122,18 +133,20 @@ Sizes sizes_of(const lazyev_t* h) {
     off += align_up((size_t)h->units * sizeof(int32_t), 256);
     const size_t qbytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
     const size_t kbytes = (size_t)h->layers * h->batch * h->kv_heads * kRowBytes;
-    s.off_q = off;
-    off += align_up(qbytes, 256);
+    s.off_q = off;                          // each staging area holds two slots
+    off += 2 * align_up(qbytes, 256);
     s.off_k = off;
-    off += align_up(kbytes, 256);
+    off += 2 * align_up(kbytes, 256);
     s.off_v = off;
-    off += align_up(kbytes, 256);
+    off += 2 * align_up(kbytes, 256);
     s.off_out = off;
-    off += align_up(qbytes, 256);
+    off += 2 * align_up(qbytes, 256);
     s.off_score = off;
     off += align_up((size_t)kScoreStageUnits * h->capacity * sizeof(double), 256);
     s.off_hist = off;
     off += align_up((size_t)kMaxHistBins * sizeof(unsigned long long), 256);
+    s.off_h2 = off;
+    off += align_up((size_t)kH2TableEntries * sizeof(double), 256);
     s.scratch = off;
     return s;
 }
@@ -202,9 +215,30 @@ int collect_profile(lazyev_t* h) {
     return LAZYEV_OK;
 }
 
-int run_evict(lazyev_t* h, int* evicted) {
+// Candidates of an eviction over n cached tokens, or -1 when the select kernel cannot hold them.
+int candidates_of(const lazyev_t* h, int n) {
+    const int ncand = n - h->n_recent - h->n_initial;
+    if (ncand <= 0 || select_smem_bytes(ncand) > 200 * 1024) return -1;
+    return ncand;
+}
+
+bool evict_due_at(const lazyev_t* h, int t, int n) { return t != 0 && t % h->window == 0 && n > h->budget_now; }
+
+// The lagged eviction of Section 4 at the current step, if one is due.  `src` and `first_moved` are
+// the work lists of the select and compact kernels: the bound scratch region's or the library's own.
+int run_evict(lazyev_t* h, int* evicted, int32_t* src, int32_t* first_moved) {
     if (evicted) *evicted = 0;
-    if (h->t == 0 || h->t % h->window != 0 || h->n <= h->budget_now) return LAZYEV_OK;
+    if (!evict_due_at(h, h->t, h->n)) return LAZYEV_OK;
+    const int ncand = candidates_of(h, h->n);
+    if (ncand < 0)
+        return fail(h, LAZYEV_EINVAL, "eviction over %d candidates is not supported", h->n - h->n_recent - h->n_initial);
+    cudaError_t e;
+    if (h->h2_table_mode != h->score_mode) {      // the H2 term per MRI value, in the variant the mode selects
+        e = h2_table_launch(h->score_mode, kH2TableEntries, h->h2_table, h->stream);
+        if (e != cudaSuccess) return cuda_fail(h, e, "H2 table launch");
+        h->h2_table_mode = h->score_mode;
+        h->launches += 1;
+    }
     EvictArgs a;
     a.n = h->n;
     a.budget = h->budget_now;
@@ -212,15 +246,14 @@ int run_evict(lazyev_t* h, int* evicted) {
     a.n_initial = h->n_initial;
     a.t = h->t;
     a.score_mode = h->score_mode;
-    a.src = h->src;
-    a.first_moved = h->first_moved;
-    if (a.n - a.n_recent - a.n_initial <= 0 || select_smem_bytes(a.n - a.n_recent - a.n_initial) > 200 * 1024)
-        return fail(h, LAZYEV_EINVAL, "eviction over %d candidates is not supported", a.n - a.n_recent - a.n_initial);
+    a.src = src;
+    a.first_moved = first_moved;
+    a.h2_table = h->h2_table;
+    a.h2_entries = kH2TableEntries;
     const Geometry geo = geometry(h);
-    cudaError_t e;
     {
         // algorithmic bytes: TS and MRI of every candidate read, the source list written
-        SpanGuard g(h, kSpanSelect, (double)h->units * (8.0 * (a.n - a.n_recent - a.n_initial) + 4.0 * a.budget));
+        SpanGuard g(h, kSpanSelect, (double)h->units * (8.0 * ncand + 4.0 * a.budget));
         e = select_launch(geo, h->st, a, h->stream);
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "select kernel launch");
@@ -229,10 +262,14 @@ int run_evict(lazyev_t* h, int* evicted) {
         e = compact_launch(geo, h->pool, h->st, a, h->stream);
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "compact kernel launch");
+    h->launches += 2;
+    h->evictions += 1;
+    if (evicted) *evicted = h->n - h->budget_now;
+    h->n = h->budget_now;
     if (h->profiling) {
         // rows that actually moved: every destination from the first evicted slot on
         std::vector<int32_t> first(h->units);
-        e = cudaMemcpyAsync(first.data(), h->first_moved, first.size() * 4, cudaMemcpyDeviceToHost, h->stream);
+        e = cudaMemcpyAsync(first.data(), first_moved, first.size() * 4, cudaMemcpyDeviceToHost, h->stream);
         if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
         if (e != cudaSuccess) return cuda_fail(h, e, "first_moved download");
         double rows = 0;
@@ -241,10 +278,6 @@ int run_evict(lazyev_t* h, int* evicted) {
         h->prof.compact_bytes += rows * (2.0 * (2 * kRowBytes + 12) + 4.0);
         h->prof.compact_rows += rows;
     }
-    h->launches += 2;
-    h->evictions += 1;
-    if (evicted) *evicted = h->n - h->budget_now;
-    h->n = h->budget_now;
     return LAZYEV_OK;
 }
 
@@ -362,6 +395,7 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
             count[ranges++] = shape.tail_units;
         }
         const size_t unit_bytes = (size_t)h->group * kRowBytes;
+        if (pipe) h->last_host_ranges = ranges;
         if (pipe) {
             for (int r = 0; r < ranges && e == cudaSuccess; ++r) {
                 e = cudaMemcpyAsync((uint8_t*)const_cast<void*>(q) + begin[r] * unit_bytes, pipe->q_host + begin[r] * unit_bytes,
@@ -419,6 +453,11 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
     if (h->n + 1 > h->capacity) return fail(h, LAZYEV_ECAPACITY, "cache full (%d slots per unit)", h->capacity);
     const int t = h->t + 1, n = h->n + 1;
+    // A step whose automatic eviction could not run is refused before anything is queued.
+    if (h->auto_evict && evict_due_at(h, t, n) && candidates_of(h, n) < 0)
+        return fail(h, LAZYEV_EINVAL,
+                    "step %d would evict over %d candidates, more than the selection supports; nothing was done", t,
+                    n - h->n_recent - h->n_initial);
     cudaError_t e;
     {
         SpanGuard g(h, kSpanAppend, 0.0);
@@ -430,7 +469,7 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     if (rc != LAZYEV_OK) return rc;
     h->t = t;
     h->n = n;
-    if (h->auto_evict) return run_evict(h, nullptr);
+    if (h->auto_evict) return run_evict(h, nullptr, h->src, h->first_moved);
     return LAZYEV_OK;
 }
 
@@ -585,12 +624,20 @@ int lazyev_bind(lazyev_t* h, void* kv_pool, void* state, void* scratch, void* cu
     uint8_t* cp = (uint8_t*)scratch;
     h->src = (int32_t*)cp;
     h->first_moved = (int32_t*)(cp + s.off_first);
-    h->stage_q = cp + s.off_q;
-    h->stage_k = cp + s.off_k;
-    h->stage_v = cp + s.off_v;
-    h->stage_out = cp + s.off_out;
+    {
+        const size_t qslot = align_up((size_t)h->layers * h->batch * h->q_heads * kRowBytes, 256);
+        const size_t kslot = align_up((size_t)h->layers * h->batch * h->kv_heads * kRowBytes, 256);
+        for (int i = 0; i < 2; ++i) {
+            h->stage_q[i] = cp + s.off_q + i * qslot;
+            h->stage_k[i] = cp + s.off_k + i * kslot;
+            h->stage_v[i] = cp + s.off_v + i * kslot;
+            h->stage_out[i] = cp + s.off_out + i * qslot;
+        }
+    }
     h->stage_score = (double*)(cp + s.off_score);
     h->stage_hist = (unsigned long long*)(cp + s.off_hist);
+    h->h2_table = (double*)(cp + s.off_h2);
+    h->h2_table_mode = -1;
 
     // Slots past n are read (and masked) by the decode kernel's last page: they must hold finite values.
     e = cudaMemsetAsync(h->pool, 0, s.kv, h->stream);
@@ -677,32 +724,58 @@ int lazyev_decode_step(lazyev_t* h, const void* q, const void* k_new, const void
     return run_step(h, q, k_new, v_new, out);
 }
 
+namespace {
+
+int host_streams(lazyev_t* h) {      // first host-buffer call: the two copy streams and their events
+    if (h->copy_in) return LAZYEV_OK;
+    cudaError_t e = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking);
+    for (int i = 0; i <= kHostChunks && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_ready, cudaEventDisableTiming);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i)
+        e = cudaEventCreateWithFlags(&h->ev_step_done[i], cudaEventDisableTiming | cudaEventBlockingSync);
+    if (e != cudaSuccess) return cuda_fail(h, e, "creating the copy streams");
+    return LAZYEV_OK;
+}
+
+// Blocks until at most `allowed` (0 or 1) asynchronous host-buffer steps are still in flight.
+int host_wait(lazyev_t* h, int allowed) {
+    cudaError_t e = cudaSuccess;
+    const int newest = (int)((h->host_seq + 1) & 1);       // slot of the step queued last
+    for (int k = 0; k < 2; ++k) {
+        const int slot = k == 0 ? newest ^ 1 : newest;      // older step first
+        if (!h->slot_busy[slot] || (allowed >= 1 && slot == newest)) continue;
+        const cudaError_t e1 = cudaEventSynchronize(h->ev_step_done[slot]);
+        if (e == cudaSuccess) e = e1;
+        h->slot_busy[slot] = false;
+    }
+    if (e != cudaSuccess) return cuda_fail(h, e, "waiting for a host-buffer step");
+    return LAZYEV_OK;
+}
+
+}  // namespace
+
 int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out) {
     if (!h) return LAZYEV_EINVAL;
     if (!q || !k_new || !v_new || !out) return fail(h, LAZYEV_EINVAL, "null pointer");
     if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
-    cudaError_t e = cudaSuccess;
-    if (!h->copy_in) {      // first call: the two copy streams and their events
-        e = cudaStreamCreateWithFlags(&h->copy_in, cudaStreamNonBlocking);
-        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_out, cudaStreamNonBlocking);
-        for (int i = 0; i <= kHostChunks && e == cudaSuccess; ++i) {
-            e = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming);
-            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming);
-        }
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_ready, cudaEventDisableTiming);
-        if (e != cudaSuccess) return cuda_fail(h, e, "creating the copy streams");
-    }
+    int rc = host_streams(h);
+    if (rc == LAZYEV_OK) rc = host_wait(h, 0);
+    if (rc != LAZYEV_OK) return rc;
     // The copy streams start after everything queued on the bound stream so far (an earlier step's
     // kernels may still read the staging buffers).
-    e = cudaEventRecord(h->ev_ready, h->stream);
+    cudaError_t e = cudaEventRecord(h->ev_ready, h->stream);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_in, h->ev_ready, 0);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_ready, 0);
     const size_t kbytes = (size_t)h->layers * h->batch * h->kv_heads * kRowBytes;
-    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_k, k_new, kbytes, cudaMemcpyHostToDevice, h->stream);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_v, v_new, kbytes, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_k[0], k_new, kbytes, cudaMemcpyHostToDevice, h->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_v[0], v_new, kbytes, cudaMemcpyHostToDevice, h->stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "host-to-device copy");
     const HostPipe pipe{(const uint8_t*)q, (uint8_t*)out};
-    const int rc = run_step(h, h->stage_q, h->stage_k, h->stage_v, h->stage_out, &pipe);
+    rc = run_step(h, h->stage_q[0], h->stage_k[0], h->stage_v[0], h->stage_out[0], &pipe);
     // both streams are drained even after an error, so that no copy is left in flight on the caller's buffers
     cudaError_t e1 = cudaStreamSynchronize(h->copy_in), e2 = cudaStreamSynchronize(h->copy_out);
     e = cudaStreamSynchronize(h->stream);
@@ -712,10 +785,87 @@ int lazyev_decode_step_host(lazyev_t* h, const void* q, const void* k_new, const
     return LAZYEV_OK;
 }
 
+int lazyev_decode_step_host_async(lazyev_t* h, const void* q, const void* k_new, const void* v_new, void* out) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!q || !k_new || !v_new || !out) return fail(h, LAZYEV_EINVAL, "null pointer");
+    if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "decode_step before prefill");
+    int rc = host_streams(h);
+    if (rc != LAZYEV_OK) return rc;
+    const int slot = (int)(h->host_seq & 1);
+    // The slot's previous step (two steps back) must be complete before its staging buffers are
+    // reused; the step before this one may still be running, and this step's uploads run beside it.
+    if (h->slot_busy[slot]) {
+        const cudaError_t e0 = cudaEventSynchronize(h->ev_step_done[slot]);
+        h->slot_busy[slot] = false;
+        if (e0 != cudaSuccess) return cuda_fail(h, e0, "waiting for a host-buffer step");
+    }
+    const size_t qbytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
+    const size_t kbytes = (size_t)h->layers * h->batch * h->kv_heads * kRowBytes;
+    cudaError_t e = cudaSuccess;
+    if (h->host_seq == 0 || !h->slot_busy[slot ^ 1]) {
+        // nothing of ours in flight: order the copy streams after whatever else the bound stream holds
+        e = cudaEventRecord(h->ev_ready, h->stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_in, h->ev_ready, 0);
+    }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_k[slot], k_new, kbytes, cudaMemcpyHostToDevice, h->copy_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_v[slot], v_new, kbytes, cudaMemcpyHostToDevice, h->copy_in);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h->stage_q[slot], q, qbytes, cudaMemcpyHostToDevice, h->copy_in);
+    if (e == cudaSuccess) e = cudaEventRecord(h->ev_in[0], h->copy_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->stream, h->ev_in[0], 0);
+    if (e != cudaSuccess) return cuda_fail(h, e, "host-to-device copy");
+    rc = run_step(h, h->stage_q[slot], h->stage_k[slot], h->stage_v[slot], h->stage_out[slot]);
+    if (rc != LAZYEV_OK) return rc;      // found before anything was queued (see lazyev_decode_step)
+    e = cudaEventRecord(h->ev_done[0], h->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_out, h->ev_done[0], 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out, h->stage_out[slot], qbytes, cudaMemcpyDeviceToHost, h->copy_out);
+    if (e == cudaSuccess) e = cudaEventRecord(h->ev_step_done[slot], h->copy_out);
+    if (e != cudaSuccess) return cuda_fail(h, e, "device-to-host copy");
+    h->slot_busy[slot] = true;
+    h->host_seq += 1;
+    return LAZYEV_OK;
+}
+
+int lazyev_host_wait(lazyev_t* h, int in_flight_allowed) {
+    if (!h) return LAZYEV_EINVAL;
+    if (in_flight_allowed < 0 || in_flight_allowed > 1) return fail(h, LAZYEV_EINVAL, "in_flight_allowed must be 0 or 1");
+    if (!h->copy_in) return LAZYEV_OK;
+    return host_wait(h, in_flight_allowed);
+}
+
+int lazyev_copy_state(lazyev_t* dst, lazyev_t* src) {
+    if (!dst || !src || dst == src) return LAZYEV_EINVAL;
+    if (!dst->bound || !src->bound) return fail(dst, LAZYEV_ESTATE, "copy_state needs two bound handles");
+    if (!src->prefilled) return fail(dst, LAZYEV_ESTATE, "copy_state from a handle that holds no cache");
+    if (dst->prefilled) return fail(dst, LAZYEV_ESTATE, "copy_state into a handle that already holds a cache (reset it first)");
+    if (dst->device != src->device || dst->layers != src->layers || dst->batch != src->batch || dst->q_heads != src->q_heads ||
+        dst->kv_heads != src->kv_heads || dst->capacity != src->capacity || dst->budget != src->budget ||
+        dst->window != src->window || dst->n_recent != src->n_recent || dst->n_initial != src->n_initial)
+        return fail(dst, LAZYEV_EINVAL, "copy_state needs two handles of the same configuration on the same device");
+    const Sizes sz = sizes_of(src);
+    cudaEvent_t ready = nullptr;
+    cudaError_t e = cudaEventCreateWithFlags(&ready, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventRecord(ready, src->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(dst->stream, ready, 0);
+    // the state region starts with the page table, so the physical pages line up with the copied pool
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dst->pool, src->pool, sz.kv, cudaMemcpyDeviceToDevice, dst->stream);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dst->st.page_table, src->st.page_table, sz.state, cudaMemcpyDeviceToDevice, dst->stream);
+    // and src's later steps must not overwrite what is still being read
+    if (e == cudaSuccess) e = cudaEventRecord(ready, dst->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(src->stream, ready, 0);
+    if (ready) cudaEventDestroy(ready);
+    if (e != cudaSuccess) return cuda_fail(dst, e, "copy_state");
+    dst->prefilled = true;
+    dst->t = src->t;
+    dst->n = src->n;
+    dst->prefill = src->prefill;
+    dst->budget_now = src->budget_now;
+    return LAZYEV_OK;
+}
+
 int lazyev_evict(lazyev_t* h, int* evicted) {
     if (!h) return LAZYEV_EINVAL;
     if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "evict before prefill");
-    return run_evict(h, evicted);
+    return run_evict(h, evicted, h->src, h->first_moved);
 }
 
 // ---- eviction without caller-provided scratch ------------------------------------------------
@@ -727,7 +877,7 @@ constexpr int kStaticMaxDevices = 64;
 static __device__ __align__(256) int32_t g_static_evict_scratch[kStaticSrcEntries + kStaticMaxUnits];
 // Device addresses of the array above, one per device ordinal.  The symbol itself is only a
 // host-side stand-in: kernels must be given the address cudaGetSymbolAddress() returns.
-static int32_t* g_static_evict_ptr[kStaticMaxDevices] = {nullptr};
+static std::atomic<int32_t*> g_static_evict_ptr[kStaticMaxDevices];
 
 int lazyev_evict_static(lazyev_t* h, int* evicted) {
     if (!h) return LAZYEV_EINVAL;
@@ -744,34 +894,28 @@ int lazyev_evict_static(lazyev_t* h, int* evicted) {
     if (dev != h->device || dev < 0 || dev >= kStaticMaxDevices)
         return fail(h, LAZYEV_ESTATE, "evict_static needs device %d (the one bound to this handle) to be current, not %d",
                     h->device, dev);
-    if (!g_static_evict_ptr[dev]) {    // first call on this device: resolve the array's device address
-        int32_t* ptr = nullptr;
-        e = cudaGetSymbolAddress((void**)&ptr, g_static_evict_scratch);
-        if (e != cudaSuccess || !ptr) return cuda_fail(h, e, "cudaGetSymbolAddress(static eviction scratch)");
-        g_static_evict_ptr[dev] = ptr;
+    int32_t* base = g_static_evict_ptr[dev].load(std::memory_order_acquire);
+    if (!base) {    // first call on this device: resolve the array's device address (threads may race; same value)
+        e = cudaGetSymbolAddress((void**)&base, g_static_evict_scratch);
+        if (e != cudaSuccess || !base) return cuda_fail(h, e, "cudaGetSymbolAddress(static eviction scratch)");
+        g_static_evict_ptr[dev].store(base, std::memory_order_release);
     }
-    if (h->t == 0 || h->t % h->window != 0 || h->n <= h->budget_now) return LAZYEV_OK;
-    EvictArgs a;
-    a.n = h->n;
-    a.budget = h->budget_now;
-    a.n_recent = h->n_recent;
-    a.n_initial = h->n_initial;
-    a.t = h->t;
-    a.score_mode = h->score_mode;
-    a.src = g_static_evict_ptr[dev];                       // every entry below budget is rewritten by the select
-    a.first_moved = g_static_evict_ptr[dev] + kStaticSrcEntries;   // kernel before the compact kernel reads it
-    const int ncand = a.n - a.n_recent - a.n_initial;
-    if (ncand <= 0 || select_smem_bytes(ncand) > 200 * 1024)
-        return fail(h, LAZYEV_EINVAL, "eviction over %d candidates is not supported", ncand);
-    const Geometry geo = geometry(h);
-    e = select_launch(geo, h->st, a, h->stream);
-    if (e != cudaSuccess) return cuda_fail(h, e, "select kernel launch");
-    e = compact_launch(geo, h->pool, h->st, a, h->stream);
-    if (e != cudaSuccess) return cuda_fail(h, e, "compact kernel launch");
-    h->launches += 2;
-    h->evictions += 1;
-    if (evicted) *evicted = h->n - h->budget_now;
-    h->n = h->budget_now;
+    // Same trigger test, kernels, timing spans and accounting as lazyev_evict(); only the work lists
+    // live elsewhere.  Every entry below budget is rewritten by the select kernel before the compact
+    // kernel reads it, so nothing in the array has to be cleared.
+    return run_evict(h, evicted, base, base + kStaticSrcEntries);
+}
+
+int lazyev_get_counters(lazyev_t* h, lazyev_counters_t* out) {
+    if (!h || !out) return LAZYEV_EINVAL;
+    if (!h->bound) return fail(h, LAZYEV_ESTATE, "get_counters before bind");
+    int32_t words[16] = {0};
+    cudaError_t e = cudaMemcpyAsync(words, h->st.status, sizeof(words), cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(h->stream);
+    if (e != cudaSuccess) return cuda_fail(h, e, "reading the device counters");
+    out->device_status = words[0];
+    out->select_radix_units = words[kCounterRadixUnits];
+    out->select_zero_cut_units = words[kCounterZeroCutUnits];
     return LAZYEV_OK;
 }
 
@@ -802,6 +946,7 @@ int lazyev_get_info(const lazyev_t* h, lazyev_info_t* out) {
     out->smem_bytes = h->last_plan.smem_bytes;
     out->launches = h->launches;
     out->evictions = h->evictions;
+    out->host_ranges = h->last_host_ranges;
     return LAZYEV_OK;
 }
 
@@ -989,6 +1134,8 @@ int lazyev_destroy(lazyev_t* h) {
         if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
     }
     if (h->ev_ready) cudaEventDestroy(h->ev_ready);
+    for (int i = 0; i < 2; ++i)
+        if (h->ev_step_done[i]) cudaEventDestroy(h->ev_step_done[i]);
     delete h;
     return LAZYEV_OK;
 }

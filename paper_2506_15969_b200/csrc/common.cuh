@@ -18,6 +18,9 @@ constexpr int kMaxGroup = 8;                       // query heads per KV head su
 // Device status word bits (state.status[0]); 0 = healthy.
 constexpr int kStatusWaitTimeout = 1;              // a bounded wait in the decode kernel gave up
 constexpr int kStatusBadIndex = 2;                 // a page / slot index was out of range
+// Words 1.. of the status array are event counters (cleared with the status word).
+constexpr int kCounterRadixUnits = 1;              // units whose selection ran the radix passes
+constexpr int kCounterZeroCutUnits = 2;            // units whose k-th score was 0: only the tie rule was left
 
 // Swizzled position of logical 16-byte chunk c (0..15) inside the row of slot r.
 __host__ __device__ __forceinline__ int swz_chunk(int c, int r) { return c ^ (r & 7); }

@@ -18,20 +18,42 @@ namespace {
 // 2 sigma(-x) is evaluated as 2 / (1 + exp(x)).
 // Modes: 0 = Eq. (2); 1 = H1 only; 2 = H2 only (the paper's ablations); 3 = Eq. (2) with
 // H2 = 2 sigma(-(MRI - 1)), a variant that decreases with MRI as the paper's prose asks.
-__device__ __forceinline__ double score_fn(int d, int mri, int mode) {
-    double h1, h2 = 0.0;
-    if (mri == 0) {
-        h1 = d == 0 ? 1.0 : 0.0;
-    } else {
-        h1 = 2.0 / (1.0 + exp((double)d / (double)mri));
-        if (mode == 3)
-            h2 = 2.0 / (1.0 + exp((double)mri - 1.0));
-        else if (mri > 1)
-            h2 = 2.0 / (1.0 + exp(1.0 / ((double)mri - 1.0)));
-    }
+__device__ __forceinline__ double h1_term(int d, int mri) {
+    if (mri == 0) return d == 0 ? 1.0 : 0.0;
+    return 2.0 / (1.0 + exp((double)d / (double)mri));
+}
+
+// The H2 term depends on MRI alone (mri >= 1 here; mode 1 never asks for it).
+__device__ __forceinline__ double h2_term(int mri, int mode) {
+    if (mode == 3) return 2.0 / (1.0 + exp((double)mri - 1.0));
+    return mri > 1 ? 2.0 / (1.0 + exp(1.0 / ((double)mri - 1.0))) : 0.0;
+}
+
+__device__ __forceinline__ double combine_terms(double h1, double h2, int mode) {
     if (mode == 1) return h1;
     if (mode == 2) return h2;
     return h1 + h2;
+}
+
+__device__ __forceinline__ double score_fn(int d, int mri, int mode) {
+    const double h1 = mode == 2 ? 0.0 : h1_term(d, mri);
+    const double h2 = (mode == 1 || mri == 0) ? 0.0 : h2_term(mri, mode);
+    return combine_terms(h1, h2, mode);
+}
+
+// The same value with the H2 term read from a table filled by h2_table_kernel with h2_term itself,
+// so both routes give identical bits.
+__device__ __forceinline__ double score_with_table(int d, int mri, int mode, const double* __restrict__ h2_table,
+                                                   int h2_entries) {
+    const double h1 = mode == 2 ? 0.0 : h1_term(d, mri);
+    double h2 = 0.0;
+    if (mode != 1 && mri != 0) h2 = mri < h2_entries ? h2_table[mri] : h2_term(mri, mode);
+    return combine_terms(h1, h2, mode);
+}
+
+__global__ void h2_table_kernel(int mode, int entries, double* table) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m < entries) table[m] = m == 0 ? 0.0 : h2_term(m, mode);
 }
 
 constexpr int kSelThreads = 512;
@@ -56,6 +78,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     __shared__ unsigned long long sh_prefix;
     __shared__ int sh_krem, sh_first, sh_done;
     __shared__ int warp_sums[kSelThreads / 32];
+    __shared__ uint32_t queue[kSelThreads / 32][64];
 
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int S = a.n_initial, R = a.n_recent;
@@ -65,14 +88,58 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     const int32_t* mri = st.mri + (size_t)u * geo.capacity + S;
     int32_t* src = a.src + (size_t)u * a.budget;
 
+    // Each warp owns a contiguous segment of the candidates and walks it 32 at a time (also in the
+    // ranking passes below, where ranks in slot order come from ballots over consecutive keys).
+    constexpr int kWarps = kSelThreads / 32;
+    const int warp = tid >> 5;
+    const int seg = ((ncand + kWarps - 1) / kWarps + 31) / 32 * 32;
+    const int seg_b = min(ncand, warp * seg), seg_e = min(ncand, seg_b + seg);
+    const unsigned lt = (1u << lane) - 1u;
+
     // Scores are >= 0, so their IEEE bit patterns order like unsigned integers; a score of exactly 0
-    // (never re-activated, the common case) has key 0.
+    // (never re-activated, the common case) has key 0.  Only re-activated tokens (MRI != 0) need the
+    // fp64 exponentials, and they are a minority scattered over the slots: a warp collects their slot
+    // numbers in a small queue and evaluates Eq. (2) for 32 of them at a time with all lanes busy,
+    // instead of every warp paying for the exponentials of its few re-activated lanes.
     int nonzero = 0;
-    for (int i = tid; i < ncand; i += kSelThreads) {
-        const unsigned long long key =
-            (unsigned long long)__double_as_longlong(score_fn(a.t - ts[i], mri[i], a.score_mode));
-        keys[i] = key;
-        nonzero += key != 0ull;
+    {
+        uint32_t* q = queue[warp];
+        int pending = 0;                           // warp-uniform
+        auto evaluate = [&](int i) {
+            const unsigned long long packed = keys[i];
+            const double sc = score_with_table((int)(packed >> 32), (int)(packed & 0xFFFFFFFFull), a.score_mode,
+                                               a.h2_table, a.h2_entries);
+            const unsigned long long key = (unsigned long long)__double_as_longlong(sc);
+            keys[i] = key;
+            nonzero += key != 0ull;
+        };
+        const unsigned long long one_bits = (unsigned long long)__double_as_longlong(1.0);
+        for (int i0 = seg_b; i0 < seg_e; i0 += 32) {
+            const int i = i0 + lane;
+            const bool in = i < seg_e;
+            const int m = in ? mri[i] : 0;
+            const int d = in ? a.t - ts[i] : 1;
+            const bool hard = in && m != 0;
+            if (in && !hard) {                     // MRI = 0: H2 = 0, H1 = 1 only at an elapsed time of 0
+                const unsigned long long key = (d == 0 && a.score_mode != 2) ? one_bits : 0ull;
+                keys[i] = key;
+                nonzero += key != 0ull;
+            }
+            if (hard) keys[i] = ((unsigned long long)(unsigned)d << 32) | (unsigned)m;
+            const unsigned mask = __ballot_sync(0xffffffffu, hard);
+            if (hard) q[pending + __popc(mask & lt)] = (uint32_t)i;
+            pending += __popc(mask);
+            __syncwarp();
+            if (pending >= 32) {
+                evaluate((int)q[lane]);
+                const uint32_t rest = lane < pending - 32 ? q[32 + lane] : 0u;
+                __syncwarp();
+                if (lane < pending - 32) q[lane] = rest;
+                pending -= 32;
+                __syncwarp();
+            }
+        }
+        if (lane < pending) evaluate((int)q[lane]);
     }
     if (tid == 0) sh_first = ncand;
     nonzero = block_sum(nonzero, warp_sums);       // (its barriers also publish keys[] and sh_first)
@@ -80,6 +147,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     // kth: bit pattern of the k-th largest score; krem: how many of the keys equal to it stay.
     unsigned long long kth = 0;
     int krem = k - nonzero;
+    if (tid == 0) atomicAdd(st.status + (nonzero > k ? kCounterRadixUnits : kCounterZeroCutUnits), 1);
     if (nonzero > k) {
         // Radix select over the non-zero keys, most significant byte first.  The histogram is built with
         // one shared-memory atomic per distinct digit and warp (scores cluster in a few exponents), and
@@ -130,13 +198,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     // keep every key > kth, and `krem` of the keys == kth
 
     // Ties are resolved towards the more recent token, i.e. the higher slot: keep the last `krem` ties.
-    // Each warp owns a contiguous segment of the candidates and walks it 32 at a time, so ranks in
-    // slot order come from ballots: lanes read consecutive keys (no bank conflicts).
-    constexpr int kWarps = kSelThreads / 32;
-    const int warp = tid >> 5;
-    const int seg = ((ncand + kWarps - 1) / kWarps + 31) / 32 * 32;
-    const int seg_b = min(ncand, warp * seg), seg_e = min(ncand, seg_b + seg);
-    const unsigned lt = (1u << lane) - 1u;
+    // Ranks in slot order come from ballots over each warp's segment: lanes read consecutive keys (no
+    // bank conflicts).
     int ties = 0;
     for (int i0 = seg_b; i0 < seg_e; i0 += 32) {
         const int i = i0 + lane;
@@ -335,6 +398,11 @@ cudaError_t select_prepare() {
 cudaError_t select_launch(const Geometry& geo, StateView st, const EvictArgs& a, cudaStream_t stream) {
     const int ncand = a.n - a.n_recent - a.n_initial;
     select_kernel<<<geo.units, kSelThreads, select_smem_bytes(ncand), stream>>>(geo, st, a);
+    return cudaGetLastError();
+}
+
+cudaError_t h2_table_launch(int score_mode, int entries, double* table, cudaStream_t stream) {
+    h2_table_kernel<<<(entries + 255) / 256, 256, 0, stream>>>(score_mode, entries, table);
     return cudaGetLastError();
 }
 

@@ -54,7 +54,13 @@ struct EvictArgs {
     int score_mode;
     int32_t* src;          // [units][budget]: slot that moves to slot j
     int32_t* first_moved;  // [units]: first j with src[j] != j (budget if none)
+    const double* h2_table;   // H2 term of the score per MRI value, for the mode in score_mode
+    int h2_entries;
 };
+
+constexpr int kH2TableEntries = 1 << 15;    // MRI values covered by the table; larger ones are evaluated directly
+// Fills table[m], m < entries, with the H2 term of Eq. (2) in the variant `score_mode` selects.
+cudaError_t h2_table_launch(int score_mode, int entries, double* table, cudaStream_t stream);
 
 size_t select_smem_bytes(int n_candidates);
 cudaError_t select_prepare();

@@ -124,7 +124,7 @@ def test_protected_tokens_and_score_variants():
                  binding.SCORE_H1_PLUS_H2_DECREASING):
         ls = lockstep(cfg, seed=4, sample_units=[0, 3, 7], score_mode=mode)
         rep = ls.run(160)
-        ls.assert_ok(jaccard=0.99)
+        ls.assert_ok()
         assert rep.evictions >= 8
         d = ls.eng.dump_state(0, 1)
         assert d["pos"][0][:4].tolist() == [0, 1, 2, 3]                 # initial tokens survive
@@ -136,7 +136,7 @@ def test_dynamic_budget_and_long_prompt():
     cfg = traces.tiny_config(budget=200, window=32, n_recent=32, prefill=150, budget_frac_tenths=3)
     ls = lockstep(cfg, seed=5, sample_units=[1, 4])
     rep = ls.run(320)
-    ls.assert_ok(jaccard=0.99)
+    ls.assert_ok()
     assert rep.evictions == 10
     assert ls.eng.info().n == cfg.budget_at(320)
 
@@ -213,7 +213,7 @@ def test_per_step_eviction_window_of_one():
     cfg = traces.tiny_config(budget=120, window=1, n_recent=1, prefill=100)
     ls = lockstep(cfg, seed=16, sample_units=[0, 2, 7])
     ls.run(90)
-    ls.assert_ok(jaccard=0.99)
+    ls.assert_ok()
     assert ls.rep.evictions == 90 - 20 and ls.eng.info().n == 120
 
 
@@ -275,7 +275,7 @@ def test_observed_prompt_then_decode(prefill):
     assert (d["mri"][0] > 0).sum() >= 5                       # prompt tokens were re-activated
     assert ls.prompt_excluded <= prefill // 25                # tokens that came within 1e-4 of the threshold
     rep = ls.run(100)
-    ls.assert_ok(jaccard=0.98)
+    ls.assert_ok()
     assert rep.evictions == 2
 
 
@@ -398,6 +398,29 @@ def test_eviction_over_too_many_candidates_is_refused():
     assert eng.info().n == 25764 and eng.dump_state()["device_status"] == 0
 
 
+def test_step_whose_automatic_eviction_cannot_run_is_refused_up_front():
+    """Automatic eviction on (the default) and a prompt beyond the selection's candidate limit: the decode
+    step at the first decision point returns EINVAL before anything is queued -- t and n do not move,
+    so the caller can retry -- instead of completing the step and then failing in the eviction."""
+    eng = binding.Engine(1, 2, 1, 128, 25700, 64, 0.5, max_prefill=25800)
+    z = torch.zeros(1, 1, 1, 25800, 128, dtype=torch.bfloat16, device="cuda")
+    eng.prefill(z, z)                                        # 25800 > budget: the step at t = 64 must evict
+    x = torch.zeros(1, 1, 2, 128, dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros(1, 1, 1, 128, dtype=torch.bfloat16, device="cuda")
+    for _ in range(63):
+        eng.decode_step(x, kv, kv, x)
+    for _ in range(2):                                       # refused twice: nothing changed in between
+        with pytest.raises(binding.LazyEvError) as e:
+            eng.decode_step(x, kv, kv, x)
+        assert e.value.code == binding.EINVAL and "candidates" in str(e.value)
+        assert (eng.info().t, eng.info().n) == (63, 25863)
+    eng.set_auto_evict(False)                                # the caller's way out: step without evicting
+    eng.decode_step(x, kv, kv, x)
+    assert (eng.info().t, eng.info().n) == (64, 25864)
+    eng.synchronize()
+    assert eng.counters().device_status == 0
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     cfg = traces.tiny_config()
     gen = traces.TraceGen(cfg, 8, device="cuda")
@@ -419,3 +442,56 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert a.info().evictions == 2 and b.info().evictions == 2          # automatic eviction ran
     for key in ("pos", "ts", "mri", "pbar"):
         assert np.array_equal(da[key], db[key])
+
+
+def test_host_buffer_pipeline_of_unit_ranges_matches_the_resident_step():
+    """1792 units: 12 full rounds of the persistent grid (split by the host-buffer entry point into
+    three unit ranges with overlapped copies) and a partly filled last round that goes to the second
+    launch.  The synchronous host call, the asynchronous host call and the resident call run side by
+    side through four evictions; outputs and all state must be identical bit for bit."""
+    from tests.harness import make_engine
+    cfg = traces.tiny_config(batch=32, layers=14, q_heads=28, kv_heads=4, prefill=1500, budget=1520, window=32,
+                             n_recent=32)
+    assert cfg.units == 1792                                 # 24 pages per unit: long enough for the second launch to pay
+    gen = traces.TraceGen(cfg, 18, device="cuda")
+    res, host, asy = make_engine(cfg), make_engine(cfg), make_engine(cfg)
+    k, v = gen.prefill()
+    shape = (cfg.layers, cfg.batch, cfg.kv_heads, cfg.prefill, 128)
+    res.prefill(k.view(shape), v.view(shape))
+    host.copy_state_from(res)                                # the fork entry point, checked by what follows
+    asy.copy_state_from(res)
+    oshape = (cfg.layers, cfg.batch, cfg.q_heads, 128)
+    out_r = torch.empty(oshape, dtype=torch.bfloat16, device="cuda")
+    out_h = torch.empty(oshape, dtype=torch.bfloat16).pin_memory()
+    out_a = [torch.empty(oshape, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    expect = [None, None]
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for chunk in range(4):                                   # 128 steps: an eviction every 32
+        q, kn, vn = gen.steps(32)
+        qh, kh, vh = q.cpu().pin_memory(), kn.cpu().pin_memory(), vn.cpu().pin_memory()
+        for s in range(32):
+            res.decode_step(q[s], kn[s], vn[s], out_r)
+            host.decode_step_host(qh[s], kh[s], vh[s], out_h)
+            ref = out_r.cpu()
+            assert torch.equal(ref, out_h), f"synchronous host step differs at chunk {chunk} step {s}"
+            i = (chunk * 32 + s) & 1
+            asy.decode_step_host_async(qh[s], kh[s], vh[s], out_a[i])
+            asy.host_wait(1)                                 # everything but the step just queued is complete
+            if expect[i ^ 1] is not None:
+                assert torch.equal(expect[i ^ 1], out_a[i ^ 1]), f"asynchronous host step differs before chunk {chunk} step {s}"
+            expect[i] = ref
+        asy.host_wait(0)
+        assert torch.equal(expect[1], out_a[1])
+        inf = host.info()
+        if sms == 148:
+            assert inf.host_ranges == 4 and inf.tail_units == 16      # three ranges of whole rounds + the last round's units
+        else:
+            assert inf.host_ranges >= 2
+    dr = res.dump_state(kv=True)
+    assert res.info().evictions == 4 and dr["n"] == cfg.budget
+    for other in (host, asy):
+        assert other.info().evictions == 4
+        do = other.dump_state(kv=True)
+        for key in ("pos", "ts", "mri", "pbar", "k", "v"):
+            assert np.array_equal(dr[key], do[key]), key
+        assert do["device_status"] == 0
