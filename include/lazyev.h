@@ -139,19 +139,52 @@ int lazyev_reset(lazyev_t* h);
  * Prompt load WITH observation.  The paper tracks recurrence while decoding and does not say
  * how TS and MRI of prompt tokens start; lazyev_prefill() takes TS = 0, MRI = 0.  This call
  * takes the other reading: tracking (Eq. 1, Algorithm 1's per-token loop) starts at the first
- * prompt token.  The prompt is loaded and then replayed through the decode kernel one row at
- * a time: row j attends causally over rows 0..j with its own queries, and the statistics are
- * updated at time j - (n_tokens - 1), so the last prompt row is time 0 and decode steps
- * continue at t = 1; a prompt token starts at TS = its own time, MRI = 0.  No eviction
- * happens during the prompt.
+ * prompt token.  Row j of the prompt attends causally over rows 0..j with its own queries
+ * (Appendix A, Eq. (attn)), every token's probability is averaged over the query heads of the
+ * group, and the statistics are updated in row order at time j - (n_tokens - 1), so the last
+ * prompt row is time 0 and decode steps continue at t = 1; a prompt token starts at TS = its
+ * own time, MRI = 0.  No eviction happens during the prompt.  The stored probabilities are
+ * those of the last prompt row.
  *   q, out : [n_tokens][layers, batch, q_heads, head_dim] bf16 (row-major by prompt position:
  *            row j is laid out like the q / out of lazyev_decode_step); out receives the
  *            causal attention output of every prompt row
  *   k, v   : as for lazyev_prefill()
- * Cost: n_tokens decode launches over 1..n_tokens cached tokens (meant for prompts of
- * hundreds to a few thousand tokens).  Errors as for lazyev_prefill().
+ * Two implementations (lazyev_set_prompt_mode): LAZYEV_PROMPT_TILED (default) is one launch of
+ * a tiled causal-attention kernel on the tensor cores that reads K / V once per tile of query
+ * rows; it wants q, k, v and out 16-byte aligned.  LAZYEV_PROMPT_REPLAY pushes the prompt
+ * through the decode kernel one row per launch (n_tokens launches over 1..n_tokens cached
+ * tokens); it is kept as a cross-check.  Their probabilities agree to float32 rounding, not
+ * bit for bit.  Errors as for lazyev_prefill(), plus EINVAL for misaligned pointers.
  */
 int lazyev_prefill_observed(lazyev_t* h, const void* q, const void* k, const void* v, int n_tokens, void* out);
+
+enum { LAZYEV_PROMPT_TILED = 0, LAZYEV_PROMPT_REPLAY = 1 };
+int lazyev_set_prompt_mode(lazyev_t* h, int mode);
+/*
+ * Diagnostics for lazyev_prefill_observed(): when device_rows != NULL the next prompt pass also
+ * writes, for units [unit_begin, unit_begin + unit_count), the group-mean probability of every
+ * token at every prompt row: device_rows[(u * n_tokens + j) * n_tokens + i] for i <= j (float32,
+ * caller-owned device memory of unit_count * n_tokens^2 floats; entries with i > j are left
+ * untouched).  NULL switches it off.  The tracking of the prompt consumes exactly these values.
+ */
+int lazyev_set_prompt_dump(lazyev_t* h, float* device_rows, int unit_begin, int unit_count);
+
+/*
+ * How long a kernel waits on one of its internal barriers (a page that never arrives, a peer
+ * block that never answers) before it gives up, sets the device status word and ends: default
+ * 2 s, settable between 0.1 ms and 60 s.  A kernel that gave up leaves the context usable;
+ * lazyev_synchronize() then returns EDEVICE and lazyev_reset() clears the word.
+ */
+int lazyev_set_wait_limit(lazyev_t* h, double seconds);
+/*
+ * Diagnostics for the time-out path (no counterpart in the paper): with pages >= 0, the warp
+ * that feeds a decode block's shared-memory page ring issues no copy beyond its first `pages`
+ * pages, so the block's other warps wait for a page that never comes, give up after the wait
+ * limit and flag the device status word.  Nothing faults: the kernel ends by itself, and the
+ * outputs and statistics of that step are undefined (lazyev_reset() before the handle is used
+ * again).  Honoured by launches with one block per unit (lazyev_set_splits(h, 1)); -1 = off.
+ */
+int lazyev_debug_starve_page_ring(lazyev_t* h, int pages);
 
 /*
  * One decode step for all units (Algorithm 1 without its last branch unless

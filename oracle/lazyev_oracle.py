@@ -257,12 +257,15 @@ class OracleUnit:
         self.MRI = np.zeros(self.P, dtype=np.int64)
         self.t = 0
 
-    def prefill_observed(self, Q, K, V) -> np.ndarray:
+    def prefill_observed(self, Q, K, V, pbar_rows=None) -> np.ndarray:
         """Prompt load with tracking from the first prompt token (the paper does not say how
         TS / MRI of prompt tokens start; this is the reading in which Algorithm 1's per-token
         loop already runs over the prompt).  Row j of the prompt attends causally over rows
         0..j at time j - (P - 1), so the last row is time 0 and decode steps go on at t = 1.
-        Q [P, G, D], K, V [P, D].  Returns the attention outputs [P, G, D]."""
+        Q [P, G, D], K, V [P, D].  Returns the attention outputs [P, G, D]; the probabilities
+        of every row are kept in `prompt_pbar` (list of arrays, row j has j + 1 entries).
+        `pbar_rows` [P, P] replaces the oracle's own probabilities in the tracking (bookkeeping
+        fed another implementation's float32 values, row j uses its first j + 1 entries)."""
         Q = np.asarray(Q, dtype=np.float64)
         K = np.asarray(K, dtype=np.float64)
         V = np.asarray(V, dtype=np.float64)
@@ -273,12 +276,11 @@ class OracleUnit:
         self.TS, self.MRI = np.zeros(0, dtype=np.int64), np.zeros(0, dtype=np.int64)
         self.t = -P                       # attend() advances t before it appends: row j runs at j - (P - 1)
         outs = np.zeros((P, self.G, self.D))
-        self.prompt_margin = np.full(P, np.inf)      # per token: closest |pbar - alpha| / alpha over the rows
+        self.prompt_pbar = []
         for j in range(P):
             outs[j], pbar = self.attend(Q[j], K[j], V[j])
-            m = np.abs(pbar - float(self.alpha32)) / max(float(self.alpha32), 1e-300)
-            self.prompt_margin[: j + 1] = np.minimum(self.prompt_margin[: j + 1], m)
-            self.track(pbar)
+            self.prompt_pbar.append(pbar)
+            self.track(pbar if pbar_rows is None else np.asarray(pbar_rows)[j, : j + 1])
         assert self.t == 0 and self.n == P
         return outs
 

@@ -17,6 +17,7 @@ from . import build as _build
 
 OK, EINVAL, ESTATE, ECAPACITY, EDEVICE, ECUDA = 0, -1, -2, -3, -4, -5
 SCORE_H1_PLUS_H2, SCORE_H1_ONLY, SCORE_H2_ONLY, SCORE_H1_PLUS_H2_DECREASING = 0, 1, 2, 3
+PROMPT_TILED, PROMPT_REPLAY = 0, 1
 
 
 class Info(C.Structure):
@@ -62,6 +63,10 @@ _PROTOS = {
     "lazyev_prefill": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int],
     "lazyev_reset": [C.c_void_p],
     "lazyev_prefill_observed": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p],
+    "lazyev_set_prompt_mode": [C.c_void_p, C.c_int],
+    "lazyev_set_prompt_dump": [C.c_void_p, C.c_void_p, C.c_int, C.c_int],
+    "lazyev_set_wait_limit": [C.c_void_p, C.c_double],
+    "lazyev_debug_starve_page_ring": [C.c_void_p, C.c_int],
     "lazyev_decode_step": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_decode_step_host": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_decode_step_host_async": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
@@ -187,6 +192,19 @@ class Engine:
 
     def reset(self) -> None:
         self._check(lib().lazyev_reset(self._h))
+
+    def set_prompt_mode(self, mode: int) -> None:
+        self._check(lib().lazyev_set_prompt_mode(self._h, mode))
+
+    def set_prompt_dump(self, rows, unit_begin: int = 0, unit_count: int = 0) -> None:
+        """lazyev_set_prompt_dump: rows = float32 CUDA tensor [unit_count, P, P] or None."""
+        self._check(lib().lazyev_set_prompt_dump(self._h, _ptr(rows), unit_begin, unit_count))
+
+    def debug_starve_page_ring(self, pages: int) -> None:
+        self._check(lib().lazyev_debug_starve_page_ring(self._h, pages))
+
+    def set_wait_limit(self, seconds: float) -> None:
+        self._check(lib().lazyev_set_wait_limit(self._h, seconds))
 
     def prefill_observed(self, q, k, v, out) -> None:
         """lazyev_prefill_observed: q, out [P, layers, batch, q_heads, D]; k, v as for prefill."""

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblazyev.so")
-SOURCES = ["api.cu", "decode.cu", "cache_ops.cu", "evict.cu"]
+SOURCES = ["api.cu", "decode.cu", "cache_ops.cu", "evict.cu", "prompt.cu"]
 
 
 def _nvcc() -> str:

@@ -24,6 +24,11 @@ struct lazyev {
     int budget = 0, budget_now = 0, window = 0, n_recent = 0, n_initial = 0, max_prefill = 0;
     float alpha = 0.f;
     int auto_evict = 1, score_mode = LAZYEV_SCORE_H1_PLUS_H2, force_splits = 0, force_stages = 0, force_groups = 0;
+    int prompt_mode = LAZYEV_PROMPT_TILED;
+    float* prompt_dump = nullptr;          // optional per-row probabilities of the prompt pass (caller's device memory)
+    int prompt_dump_begin = 0, prompt_dump_count = 0;
+    unsigned long long wait_limit_ns = 2000000000ull;   // bounded waits in the kernels give up after this long
+    int stop_after_pages = -1;             // diagnostics: starve the decode kernel's page ring (-1: off)
     // derived at bind
     bool bound = false, prefilled = false;
     int units = 0, group = 0, capacity = 0, pages_per_unit = 0;
@@ -292,7 +297,8 @@ struct HostPipe {
 // tracking at time t.
 int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPipe* pipe) {
     cudaError_t e = cudaSuccess;
-    DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages, h->force_groups};
+    DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages, h->force_groups,
+                   h->wait_limit_ns, h->stop_after_pages};
     // Launch shape, chosen per number of pages in use and cached.  For every cluster size whose logits
     // fit, a small time model gives the time of the rounds of the round-robin walk; the main launch is
     // the size with the least total.  A partly filled last round goes to a second launch with larger
@@ -422,7 +428,8 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
             const bool is_tail = shape.tail_units > 0 && r == ranges - 1;
             if (pipe) e = cudaStreamWaitEvent(h->stream, h->ev_in[r], 0);
             if (e != cudaSuccess) break;
-            DecodeArgs a{h->pool, h->st, q, out, n, t, begin[r], count[r]};
+            // a range of the main walk continues it; the last round's units are a walk of their own
+            DecodeArgs a{h->pool, h->st, q, out, n, t, begin[r], count[r], is_tail ? 0 : begin[r] / clusters};
             const bool beside = is_tail && fork;
             if (e != cudaSuccess) break;
             e = decode_launch(c, is_tail ? tail_plan : plan, is_tail ? count[r] : (clusters < count[r] ? clusters : count[r]), a,
@@ -701,20 +708,78 @@ int lazyev_prefill_observed(lazyev_t* h, const void* q, const void* k, const voi
     if (h->prefilled) return fail(h, LAZYEV_ESTATE, "prefill called twice");
     if (!q || !k || !v || !out || n_tokens <= 0) return fail(h, LAZYEV_EINVAL, "null pointer or non-positive token count");
     if (n_tokens > h->max_prefill) return fail(h, LAZYEV_ECAPACITY, "prompt of %d tokens exceeds max_prefill = %d", n_tokens, h->max_prefill);
-    // rows are loaded with TS = their own time j - (P - 1) <= 0, then replayed through the decode kernel
+    if (h->prompt_mode == LAZYEV_PROMPT_TILED && (((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15))
+        return fail(h, LAZYEV_EINVAL, "q, k, v and out must be 16-byte aligned");
+    // rows are loaded with TS = their own time j - (P - 1) <= 0 and MRI = 0
     cudaError_t e = prefill_launch(geometry(h), h->pool, h->st, k, v, n_tokens, 1 - n_tokens, h->stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "prefill kernel launch");
     h->launches += 1;
-    const size_t row_bytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
-    for (int j = 0; j < n_tokens; ++j) {
-        const int rc = run_decode(h, (const uint8_t*)q + j * row_bytes, (uint8_t*)out + j * row_bytes, j + 1,
-                                  j - (n_tokens - 1), nullptr);
-        if (rc != LAZYEV_OK) return rc;
+    if (h->prompt_mode == LAZYEV_PROMPT_TILED) {
+        // one launch: tiled causal attention on the tensor cores, K / V read once per query tile
+        PromptArgs a;
+        a.q = q;
+        a.k = k;
+        a.v = v;
+        a.out = out;
+        a.n_tokens = n_tokens;
+        a.alpha = h->alpha;
+        a.dump = h->prompt_dump;
+        a.dump_begin = h->prompt_dump_begin;
+        a.dump_count = h->prompt_dump_count;
+        a.wait_limit_ns = h->wait_limit_ns;
+        e = prompt_launch(geometry(h), h->st, a, h->num_sms, h->stream);
+        if (e != cudaSuccess) return cuda_fail(h, e, "prompt kernel launch");
+        h->launches += 1;
+    } else {
+        // the prompt replayed through the decode kernel, one row per launch
+        const size_t row_bytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
+        for (int j = 0; j < n_tokens; ++j) {
+            const int rc = run_decode(h, (const uint8_t*)q + j * row_bytes, (uint8_t*)out + j * row_bytes, j + 1,
+                                      j - (n_tokens - 1), nullptr);
+            if (rc != LAZYEV_OK) return rc;
+            if (h->prompt_dump) {    // row j of the per-row probabilities: tokens 0 .. j of the dumped units
+                e = cudaMemcpy2DAsync(h->prompt_dump + (size_t)j * n_tokens, (size_t)n_tokens * n_tokens * sizeof(float),
+                                      h->st.pbar + (size_t)h->prompt_dump_begin * h->capacity, (size_t)h->capacity * sizeof(float),
+                                      (size_t)(j + 1) * sizeof(float), h->prompt_dump_count, cudaMemcpyDeviceToDevice, h->stream);
+                if (e != cudaSuccess) return cuda_fail(h, e, "prompt probability dump");
+            }
+        }
     }
     h->prefilled = true;
     h->prefill = n_tokens;
     h->n = n_tokens;
     h->t = 0;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_prompt_mode(lazyev_t* h, int mode) {
+    if (!h) return LAZYEV_EINVAL;
+    if (mode != LAZYEV_PROMPT_TILED && mode != LAZYEV_PROMPT_REPLAY) return fail(h, LAZYEV_EINVAL, "unknown prompt mode %d", mode);
+    h->prompt_mode = mode;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_prompt_dump(lazyev_t* h, float* device_rows, int unit_begin, int unit_count) {
+    if (!h) return LAZYEV_EINVAL;
+    if (device_rows && (unit_begin < 0 || unit_count <= 0 || unit_begin + unit_count > h->units))
+        return fail(h, LAZYEV_EINVAL, "unit range out of bounds");
+    h->prompt_dump = device_rows;
+    h->prompt_dump_begin = device_rows ? unit_begin : 0;
+    h->prompt_dump_count = device_rows ? unit_count : 0;
+    return LAZYEV_OK;
+}
+
+int lazyev_debug_starve_page_ring(lazyev_t* h, int pages) {
+    if (!h) return LAZYEV_EINVAL;
+    if (pages < -1) return fail(h, LAZYEV_EINVAL, "pages must be -1 (off) or >= 0");
+    h->stop_after_pages = pages;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_wait_limit(lazyev_t* h, double seconds) {
+    if (!h) return LAZYEV_EINVAL;
+    if (!(seconds >= 1e-4 && seconds <= 60.0)) return fail(h, LAZYEV_EINVAL, "wait limit must be between 0.1 ms and 60 s");
+    h->wait_limit_ns = (unsigned long long)(seconds * 1e9);
     return LAZYEV_OK;
 }
 

@@ -62,16 +62,18 @@ struct DecodeParams {
     float alpha, scale_log2, inv_group;
     int splits, stages, pages_per_cta, logit_stride, tmem_pages, tmem_cols;
     int off_logits, off_xchg, off_wml, off_slots, off_misc, off_bars;
+    unsigned long long wait_limit_ns;               // a wait that lasts this long is a failure, not a delay
+    int stop_after_pages;                           // diagnostics: the producer issues no copy beyond this many (-1: off)
+    int rounds_before;                              // rounds of the round-robin walk that earlier launches of this step took
 };
 
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s is a failure, not a delay
 constexpr float kRaiseMargin = 8.f;                // log2 units a logit may exceed the softmax reference by
 
 // Bounded wait on an mbarrier phase.  On time-out the block-wide abort flag and
 // the device status word are set; once the flag is up no wait blocks any more,
 // so that every thread still reaches the cluster barriers and the kernel ends.
 __device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                           bool honour_abort = true) {
+                                           unsigned long long limit_ns, bool honour_abort = true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (honour_abort && *abort_flag) return false;
     uint32_t spins = 0;
@@ -82,7 +84,7 @@ __device__ __forceinline__ bool wait_phase(uint64_t* bar, uint32_t parity, volat
             const uint64_t now = global_timer_ns();
             if (t_start == 0) {
                 t_start = now;
-            } else if (now - t_start > kWaitLimitNs) {
+            } else if (now - t_start > limit_ns) {
                 *abort_flag = 1;
                 atomicOr(status, kStatusWaitTimeout);
                 return false;
@@ -154,14 +156,21 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         // ------------------------------------------------------------ producer
         uint32_t pc = 0, stage = 0, parity = 1;     // parity of the "empty" phase that frees the stage
         int it = 0;
-        for (int u = p.unit_begin + cluster_id; u < p.unit_end; u += n_clusters, ++it) {
+        bool stopped = false;
+        for (int u = p.unit_begin + cluster_id; u < p.unit_end && !stopped; u += n_clusters, ++it) {
             const int32_t* pt = p.page_table + (size_t)u * p.pages_per_unit + pg0;
-            for (int base = 0; base < npg; base += 32) {
+            for (int base = 0; base < npg && !stopped; base += 32) {
                 const int cnt = min(32, npg - base);
                 const int32_t entry = lane < cnt ? pt[base + lane] : 0;
                 for (int j = 0; j < cnt; ++j, ++pc) {
+                    // Diagnostics (one block per unit only): stop feeding the ring, so that the consumers'
+                    // bounded waits run out.  Every copy issued so far was armed, so the drain below is exact.
+                    if (!clustered && p.stop_after_pages >= 0 && pc >= (uint32_t)p.stop_after_pages) {
+                        stopped = true;
+                        break;
+                    }
                     int32_t pp = __shfl_sync(0xffffffffu, entry, j);
-                    if (pc >= (uint32_t)NS) wait_phase(&empty[stage], parity, abort_flag, p.status);
+                    if (pc >= (uint32_t)NS) wait_phase(&empty[stage], parity, abort_flag, p.status, p.wait_limit_ns);
                     if (lane == 0) {
                         if (pp < 0 || pp >= p.total_pages) {
                             atomicOr(p.status, kStatusBadIndex);
@@ -184,10 +193,10 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
             }
         }
         if (clustered && it > 0) cluster_wait();
-        if (*abort_flag) {   // consumers stopped waiting: let the copies in flight land before the block exits
+        if (*abort_flag || stopped) {   // consumers stopped waiting: let the copies in flight land before the block exits
             const uint32_t last = pc < (uint32_t)NS ? pc : (uint32_t)NS;
             for (uint32_t k = pc - last; k < pc; ++k)
-                wait_phase(&full[k % NS], (k / NS) & 1, abort_flag, p.status, false);
+                wait_phase(&full[k % NS], (k / NS) & 1, abort_flag, p.status, p.wait_limit_ns, false);
         }
     } else {
         // ------------------------------------------------------------ consumers
@@ -222,7 +231,11 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         const uint32_t pc_total = (uint32_t)my_units * (uint32_t)npg;
         const int tok0 = pg0 * kPageTokens;           // first token of this block's chunk
         uint32_t pc_base = 0;                         // pages of this block before the current unit
-        uint32_t pc_mod = 0;                          // pc_base mod NG
+        // Which group takes which page of a unit depends on how many pages the block has seen before it;
+        // the order in which the partial sums are added follows from that.  When the walk over the units
+        // is split over several launches, a launch starts where the one before it left off, so that every
+        // unit gets the same bits whichever launch it falls into.
+        uint32_t pc_mod = (uint32_t)(((long long)p.rounds_before * npg) % NG);   // pages before the current unit, mod NG
         uint32_t st_base = 0;                         // ring stage of page pc_base
         uint32_t pc_seen = 0, st_seen = 0, par_seen = 0;   // next page whose "full" phase this warp observes
         float lse0 = 0.f, lse1 = 0.f;                 // log-sum-exp of the previous unit, heads h0 and h1
@@ -233,7 +246,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         // wait is only valid for a waiter that saw the previous phase of that barrier.
         auto observe_through = [&](uint32_t last) {
             while (pc_seen <= last && pc_seen < pc_total) {
-                wait_phase(&full[st_seen], par_seen, abort_flag, p.status);
+                wait_phase(&full[st_seen], par_seen, abort_flag, p.status, p.wait_limit_ns);
                 ++pc_seen;
                 if (++st_seen == (uint32_t)NS) {
                     st_seen = 0;
@@ -726,6 +739,9 @@ cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clu
     p.off_slots = plan.off_slots;
     p.off_misc = plan.off_misc;
     p.off_bars = plan.off_bars;
+    p.wait_limit_ns = c.wait_limit_ns;
+    p.stop_after_pages = c.stop_after_pages;
+    p.rounds_before = a.rounds_before;
     return plan.groups == 2 ? launch_impl<2>(p, plan, clusters, stream, nullptr)
                             : launch_impl<1>(p, plan, clusters, stream, nullptr);
 }

@@ -78,7 +78,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     __shared__ unsigned long long sh_prefix;
     __shared__ int sh_krem, sh_first, sh_done;
     __shared__ int warp_sums[kSelThreads / 32];
-    __shared__ uint32_t queue[kSelThreads / 32][64];
 
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     const int S = a.n_initial, R = a.n_recent;
@@ -97,49 +96,28 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     const unsigned lt = (1u << lane) - 1u;
 
     // Scores are >= 0, so their IEEE bit patterns order like unsigned integers; a score of exactly 0
-    // (never re-activated, the common case) has key 0.  Only re-activated tokens (MRI != 0) need the
-    // fp64 exponentials, and they are a minority scattered over the slots: a warp collects their slot
-    // numbers in a small queue and evaluates Eq. (2) for 32 of them at a time with all lanes busy,
-    // instead of every warp paying for the exponentials of its few re-activated lanes.
+    // (never re-activated) has key 0.  Whether a score is exactly 0 follows from the integers alone:
+    // with MRI = 0 it is 0 unless the elapsed time is 0; with MRI != 0 the H1 term 2 / (1 + exp(d / MRI))
+    // is positive as long as the exponential is finite (d / MRI <= 700 is far inside that range; beyond
+    // it the score is evaluated to see); H2 alone (mode 2) is 0 exactly for MRI <= 1.  So the first pass
+    // needs no floating point: it stores 0 or the packed pair (d, MRI) with the top bit set, and counts.
     int nonzero = 0;
-    {
-        uint32_t* q = queue[warp];
-        int pending = 0;                           // warp-uniform
-        auto evaluate = [&](int i) {
-            const unsigned long long packed = keys[i];
-            const double sc = score_with_table((int)(packed >> 32), (int)(packed & 0xFFFFFFFFull), a.score_mode,
-                                               a.h2_table, a.h2_entries);
-            const unsigned long long key = (unsigned long long)__double_as_longlong(sc);
-            keys[i] = key;
-            nonzero += key != 0ull;
-        };
-        const unsigned long long one_bits = (unsigned long long)__double_as_longlong(1.0);
-        for (int i0 = seg_b; i0 < seg_e; i0 += 32) {
-            const int i = i0 + lane;
-            const bool in = i < seg_e;
-            const int m = in ? mri[i] : 0;
-            const int d = in ? a.t - ts[i] : 1;
-            const bool hard = in && m != 0;
-            if (in && !hard) {                     // MRI = 0: H2 = 0, H1 = 1 only at an elapsed time of 0
-                const unsigned long long key = (d == 0 && a.score_mode != 2) ? one_bits : 0ull;
-                keys[i] = key;
-                nonzero += key != 0ull;
-            }
-            if (hard) keys[i] = ((unsigned long long)(unsigned)d << 32) | (unsigned)m;
-            const unsigned mask = __ballot_sync(0xffffffffu, hard);
-            if (hard) q[pending + __popc(mask & lt)] = (uint32_t)i;
-            pending += __popc(mask);
-            __syncwarp();
-            if (pending >= 32) {
-                evaluate((int)q[lane]);
-                const uint32_t rest = lane < pending - 32 ? q[32 + lane] : 0u;
-                __syncwarp();
-                if (lane < pending - 32) q[lane] = rest;
-                pending -= 32;
-                __syncwarp();
-            }
+    for (int i0 = seg_b; i0 < seg_e; i0 += 32) {
+        const int i = i0 + lane;
+        if (i < seg_e) {
+            const int m = mri[i], d = a.t - ts[i];
+            bool zero;
+            if (a.score_mode == 2)
+                zero = m <= 1;
+            else if (m == 0)
+                zero = d != 0;
+            else if ((long long)d > 700ll * m)
+                zero = score_with_table(d, m, a.score_mode, a.h2_table, a.h2_entries) == 0.0;
+            else
+                zero = false;
+            keys[i] = zero ? 0ull : (1ull << 63) | ((unsigned long long)(unsigned)d << 32) | (unsigned)m;
+            nonzero += !zero;
         }
-        if (lane < pending) evaluate((int)q[lane]);
     }
     if (tid == 0) sh_first = ncand;
     nonzero = block_sum(nonzero, warp_sums);       // (its barriers also publish keys[] and sh_first)
@@ -149,7 +127,16 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     int krem = k - nonzero;
     if (tid == 0) atomicAdd(st.status + (nonzero > k ? kCounterRadixUnits : kCounterZeroCutUnits), 1);
     if (nonzero > k) {
-        // Radix select over the non-zero keys, most significant byte first.  The histogram is built with
+        // More non-zero scores than tokens to keep: the k-th score has to be found.  Eq. (2) in fp64 for
+        // every non-zero candidate (most of them in this regime, so the warps stay converged) ...
+        for (int i = tid; i < ncand; i += kSelThreads) {
+            const unsigned long long packed = keys[i];
+            if (packed != 0ull)
+                keys[i] = (unsigned long long)__double_as_longlong(score_with_table(
+                    (int)((packed >> 32) & 0x7FFFFFFFull), (int)(packed & 0xFFFFFFFFull), a.score_mode, a.h2_table, a.h2_entries));
+        }
+        __syncthreads();
+        // ... then a radix select over the non-zero keys, most significant byte first.  The histogram is built with
         // one shared-memory atomic per distinct digit and warp (scores cluster in a few exponents), and
         // the passes stop as soon as the k-th key is alone in its bin.
         unsigned long long prefix = 0, mask = 0;

@@ -12,6 +12,8 @@ struct DecodeConfig {
     int force_splits;      // 0 = automatic
     int force_stages;      // 0 = automatic
     int force_groups;      // 0 = automatic; groups of four consumer warps per block (1 or 2)
+    unsigned long long wait_limit_ns;   // bounded waits give up after this long
+    int stop_after_pages;  // diagnostics: -1 = off
 };
 
 struct DecodePlan {
@@ -27,6 +29,7 @@ struct DecodeArgs {
     int n;                 // cached tokens per unit, the new one included
     int t;                 // this decode step
     int unit_begin, unit_count;   // the units this launch covers
+    int rounds_before;            // whole rounds of the same walk done by earlier launches (0 for a walk of its own)
 };
 
 // Deepest ring and the shared-memory layout for n cached tokens and a cluster of `splits` blocks;
@@ -44,6 +47,21 @@ cudaError_t prefill_launch(const Geometry& geo, uint8_t* pool, StateView st, con
                            int n_tokens, int ts_first, cudaStream_t stream);
 cudaError_t append_launch(const Geometry& geo, uint8_t* pool, StateView st, const void* k_new, const void* v_new,
                           int slot, int t, int position, cudaStream_t stream);
+
+// ---- prompt pass (causal attention over the prompt with tracking) -----------------------------------
+struct PromptArgs {
+    const void* q;         // [P][units][group][128] bf16
+    const void* k;         // [units][P][128] bf16
+    const void* v;
+    void* out;             // like q
+    int n_tokens;          // P
+    float alpha;
+    float* dump;           // optional [dump_count][P][P] probabilities per prompt row
+    int dump_begin, dump_count;
+    unsigned long long wait_limit_ns;
+};
+// TS / MRI of the prompt tokens must already hold their starting values (TS = own time, MRI = 0).
+cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a, int num_sms, cudaStream_t stream);
 
 // ---- eviction --------------------------------------------------------------------
 struct EvictArgs {

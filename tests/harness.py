@@ -58,7 +58,8 @@ def make_oracle(cfg: traces.TraceConfig, score_mode="h1+h2") -> orc.OracleUnit:
 class Lockstep:
     def __init__(self, cfg: traces.TraceConfig, seed: int, sample_units, splits: int = 0, stages: int = 0,
                  score_mode: int = 0, page_table=None, pure: bool = True, check_inputs: bool = True,
-                 groups: int = 0, observed: bool = False, gen_device: str = "cuda", pure_units=None):
+                 groups: int = 0, observed: bool = False, gen_device: str = "cuda", pure_units=None,
+                 prompt_mode: int = 0):
         """`gen_device`: where the trace of all units is generated ("cpu": generated on the host and
         uploaded, so that the library's kernels are the only ones launched).  `pure_units`: the sampled
         units that also get a pure-oracle run (default: all of them, when `pure`)."""
@@ -75,6 +76,8 @@ class Lockstep:
             self.eng.set_score_mode(score_mode)
         if page_table is not None:
             self.eng.set_page_table(page_table)
+        if prompt_mode:
+            self.eng.set_prompt_mode(prompt_mode)
         mode = orc.SCORE_MODES[score_mode]
         self.gen_gpu = traces.TraceGen(cfg, seed, device=gen_device)
         self.gen_cpu = traces.TraceGen(cfg, seed, device="cpu", units=self.sample)
@@ -105,8 +108,10 @@ class Lockstep:
 
     def _observed_prefill(self, kk, vv, kc, vc, seed):
         """Prompt load with tracking: seeded prompt queries, some rows re-aligned with earlier keys so
-        that prompt tokens are re-activated; GPU against the oracle, then the shadow adopts the GPU's
-        TS / MRI (they may differ only where a probability came within 1e-4 (relative) of the threshold)."""
+        that prompt tokens are re-activated.  The library also dumps the probabilities of every prompt
+        row for the sampled units; the shadow oracle's tracking consumes them (as it does in the decode
+        steps), so TS and MRI of every prompt token must match bit for bit, while outputs and
+        probabilities are compared with the oracle's own within the tolerances."""
         cfg, P = self.cfg, self.cfg.prefill
         g = torch.Generator().manual_seed(1000 + seed)
         q = torch.randn(P, cfg.units, cfg.group, cfg.head_dim, generator=g)
@@ -118,26 +123,32 @@ class Lockstep:
                 q[j, u] += 4.0 * (cfg.head_dim ** 0.5) * kf[u, i] / kf[u, i].pow(2).sum()
         q = q.to(torch.bfloat16)
         out = torch.empty(P, cfg.units, cfg.group, cfg.head_dim, dtype=torch.bfloat16, device="cuda")
+        u0, u1 = min(self.sample), max(self.sample) + 1
+        rows_gpu = torch.zeros(u1 - u0, P, P, dtype=torch.float32, device="cuda")
+        self.eng.set_prompt_dump(rows_gpu, u0, u1 - u0)
         self.eng.prefill_observed(q.cuda(), kk, vv, out)
+        self.eng.set_prompt_dump(None)
+        rows_gpu = rows_gpu.cpu().numpy()
         rep = self.rep
-        self.prompt_excluded = 0
+        a32 = np.float32(cfg.threshold)
         for i, u in enumerate(self.sample):
             sh = self.shadow[i]
-            ref = sh.prefill_observed(f64(q[:, u]), f64(kc[i]), f64(vc[i]))
+            ref = sh.prefill_observed(f64(q[:, u]), f64(kc[i]), f64(vc[i]), pbar_rows=rows_gpu[u - u0])
             if self.pure and self.pure[i]:
                 self.pure[i].prefill_observed(f64(q[:, u]), f64(kc[i]), f64(vc[i]))
             got = f64(out[:, u])
             rep.max_out_err = max(rep.max_out_err, float((np.abs(got - ref) / (OUT_ATOL + OUT_RTOL * np.abs(ref))).max()))
+            for j in range(P):
+                mine, theirs = sh.prompt_pbar[j], rows_gpu[u - u0, j, : j + 1]
+                rep.max_pbar_err = max(rep.max_pbar_err, float(np.abs(theirs - mine).max()))
+                rep.threshold_flips += int(((mine.astype(np.float32) >= a32) != (theirs >= a32)).sum())
             d = self._dump(u)
             assert d["n"] == P and d["t"] == 0
-            rep.max_pbar_err = max(rep.max_pbar_err, float(np.abs(d["pbar"][0] - sh.last_pbar).max()))
-            clear = sh.prompt_margin > 1e-4
-            assert np.array_equal(d["ts"][0][clear], sh.TS[clear]), f"prompt TS mismatch unit {u}"
-            assert np.array_equal(d["mri"][0][clear], sh.MRI[clear]), f"prompt MRI mismatch unit {u}"
+            assert np.array_equal(d["pbar"][0], rows_gpu[u - u0, P - 1]), "stored probabilities are not the last row's"
+            assert np.array_equal(d["ts"][0], sh.TS), f"prompt TS mismatch unit {u}"
+            assert np.array_equal(d["mri"][0], sh.MRI), f"prompt MRI mismatch unit {u}"
             assert np.array_equal(d["pos"][0], sh.pos)
-            self.prompt_excluded += int((~clear).sum())
             rep.activations += int((sh.MRI > 0).sum())
-            sh.TS, sh.MRI = d["ts"][0].astype(np.int64), d["mri"][0].astype(np.int64)
 
     def _dump(self, u, **kw):
         return self.eng.dump_state(u, 1, **kw)
