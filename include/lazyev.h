@@ -283,7 +283,9 @@ int lazyev_evict(lazyev_t* h, int* evicted);
  * handle gets LAZYEV_ECAPACITY and a message naming both numbers, before anything runs.
  * The device bound to the handle must be the current device (ESTATE otherwise).
  * The first call on each device looks up the array's device address (one
- * cudaGetSymbolAddress call, no allocation); make that first call outside any stream capture.
+ * cudaGetSymbolAddress call; the CUDA runtime may load the library's static data at that moment,
+ * which is when the 4 MiB show up in the device's memory in use); make that first call outside
+ * any stream capture.  Later calls leave the amount of device memory in use unchanged.
  * All handles and all calls on one GPU share the one array and it keeps whatever the last
  * call left in it.  Nothing in it has to start at zero: the select kernel rewrites every entry
  * that the compact kernel reads.  Two evict_static calls whose kernels overlap on the GPU
@@ -409,6 +411,11 @@ int lazyev_synchronize(lazyev_t* h);
 
 /* Frees the host-side handle.  Device memory stays with the caller. */
 int lazyev_destroy(lazyev_t* h);
+
+/* Bit 0: the library was compiled with -DLAZYEV_DEBUG_BOUNDS: every slot, page-table and work-list
+ * index in the kernels is range-checked, a failed check sets bit 1 of the device status word and the
+ * access is skipped (slower; for tests -- the release build has none of these checks). */
+int lazyev_build_flags(void);
 
 const char* lazyev_strerror(int code);
 const char* lazyev_last_error(const lazyev_t* h);

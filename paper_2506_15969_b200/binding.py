@@ -89,12 +89,20 @@ _PROTOS = {
 _lib = None
 
 
+def debug_bounds_requested() -> bool:
+    """LAZYEV_DEBUG_BOUNDS=1 in the environment selects the range-checked build of the library."""
+    return os.environ.get("LAZYEV_DEBUG_BOUNDS", "0") == "1"
+
+
 def lib() -> C.CDLL:
     """Load (building first if the sources are newer) the shared library."""
     global _lib
     if _lib is None:
-        path = _build.build()
+        path = _build.build(debug_bounds=debug_bounds_requested())
         _lib = C.CDLL(path)
+        _lib.lazyev_build_flags.argtypes, _lib.lazyev_build_flags.restype = [], C.c_int
+        if bool(_lib.lazyev_build_flags() & 1) != debug_bounds_requested():
+            raise RuntimeError(f"{path} is not the build flavour that was asked for")
         for name, args in _PROTOS.items():
             fn = getattr(_lib, name)
             fn.argtypes, fn.restype = args, C.c_int

@@ -498,6 +498,8 @@ const char* lazyev_strerror(int code) {
 
 const char* lazyev_last_error(const lazyev_t* h) { return h ? h->err : "null handle"; }
 
+int lazyev_build_flags(void) { return kBuildFlags; }
+
 int lazyev_create(lazyev_t** handle, int layers, int q_heads, int kv_heads, int head_dim, int budget, int window,
                   float threshold) {
     if (!handle) return LAZYEV_EINVAL;

@@ -29,7 +29,9 @@ __global__ void prefill_kernel(Geometry geo, uint8_t* pool, StateView st, const 
     const size_t total = (size_t)geo.units * n_tokens;
     for (size_t w = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; w < total; w += warps) {
         const int u = (int)(w / n_tokens), i = (int)(w % n_tokens);
+        if (!in_bounds(i < geo.capacity, st.status)) continue;
         const int32_t pp = st.page_table[(size_t)u * geo.pages_per_unit + i / kPageTokens];
+        if (!in_bounds(pp >= 0 && pp < geo.units * geo.pages_per_unit, st.status)) continue;
         const int r = i % kPageTokens, c = lane & 15;
         const uint4* src = (lane < 16 ? k : v) + w * kChunksPerRow + c;
         uint8_t* row = page_ptr(pool, pp) + (lane < 16 ? 0 : kPageHalfBytes) + r * kRowBytes;
@@ -51,7 +53,9 @@ __global__ void append_kernel(Geometry geo, uint8_t* pool, StateView st, const u
     const int lane = threadIdx.x & 31;
     const int u = (int)(((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
     if (u >= geo.units) return;
+    if (!in_bounds(slot >= 0 && slot < geo.capacity, st.status)) return;
     const int32_t pp = st.page_table[(size_t)u * geo.pages_per_unit + slot / kPageTokens];
+    if (!in_bounds(pp >= 0 && pp < geo.units * geo.pages_per_unit, st.status)) return;
     const int r = slot % kPageTokens, c = lane & 15;
     const uint4* src = (lane < 16 ? k_new : v_new) + (size_t)u * kChunksPerRow + c;
     uint8_t* row = page_ptr(pool, pp) + (lane < 16 ? 0 : kPageHalfBytes) + r * kRowBytes;

@@ -22,6 +22,19 @@ constexpr int kStatusBadIndex = 2;                 // a page / slot index was ou
 constexpr int kCounterRadixUnits = 1;              // units whose selection ran the radix passes
 constexpr int kCounterZeroCutUnits = 2;            // units whose k-th score was 0: only the tie rule was left
 
+// Index checks of the debug build (-DLAZYEV_DEBUG_BOUNDS): a failed check flags the status word and
+// the caller skips the access.  In the release build the checks compile to nothing.
+#ifdef LAZYEV_DEBUG_BOUNDS
+__device__ __forceinline__ bool in_bounds(bool ok, int32_t* status) {
+    if (!ok) atomicOr(status, kStatusBadIndex);
+    return ok;
+}
+constexpr int kBuildFlags = 1;
+#else
+__device__ __forceinline__ bool in_bounds(bool, int32_t*) { return true; }
+constexpr int kBuildFlags = 0;
+#endif
+
 // Swizzled position of logical 16-byte chunk c (0..15) inside the row of slot r.
 __host__ __device__ __forceinline__ int swz_chunk(int c, int r) { return c ^ (r & 7); }
 

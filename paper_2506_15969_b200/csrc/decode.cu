@@ -261,6 +261,10 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 tmem_wait_ld();
             } else {
                 const int i = (j - tmem_pages) * kPageTokens + (int)tok_off + g;
+                if (!in_bounds(i >= 0 && i + 8 < LS, p.status)) {
+                    x00 = x01 = x10 = x11 = 0.f;
+                    return;
+                }
                 x00 = h0_on ? spill[h0 * LS + i] : 0.f;
                 x10 = h0_on ? spill[h0 * LS + i + 8] : 0.f;
                 x01 = h1_on ? spill[h1 * LS + i] : 0.f;
@@ -272,6 +276,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 tmem_st4(tmem_lane + 4 * j, x00, x01, x10, x11);
             } else {
                 const int i = (j - tmem_pages) * kPageTokens + (int)tok_off + g;
+                if (!in_bounds(i >= 0 && i + 8 < LS, p.status)) return;
                 if (h0_on) {
                     spill[h0 * LS + i] = x00;
                     spill[h0 * LS + i + 8] = x10;
@@ -317,6 +322,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                 retire_pending();
                 const size_t row = (size_t)u_prev * p.capacity + tok0;
                 const int i0 = base + g, i1 = base + g + 8;
+                if (!in_bounds(u_prev >= p.unit_begin && u_prev < p.unit_end && p.n <= p.capacity, p.status)) return;
                 if (tok0 + i0 < p.n) {
                     const float pb = a0 * p.inv_group;
                     p.pbar[row + i0] = pb;

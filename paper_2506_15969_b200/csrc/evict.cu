@@ -86,6 +86,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     const int32_t* ts = st.ts + (size_t)u * geo.capacity + S;
     const int32_t* mri = st.mri + (size_t)u * geo.capacity + S;
     int32_t* src = a.src + (size_t)u * a.budget;
+    if (!in_bounds(S >= 0 && R >= 0 && ncand > 0 && k >= 0 && k <= ncand && a.n <= geo.capacity && a.budget <= a.n, st.status))
+        return;
 
     // Each warp owns a contiguous segment of the candidates and walks it 32 at a time (also in the
     // ranking passes below, where ranks in slot order come from ballots over consecutive keys).
@@ -232,7 +234,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
             const int i = i0 + lane;
             const bool keep = (keep_bits >> step) & 1ull;
             const unsigned keep_mask = __ballot_sync(0xffffffffu, keep);
-            if (keep) src[S + dst + __popc(keep_mask & lt)] = S + i;
+            if (keep && in_bounds(S + dst + __popc(keep_mask & lt) < a.budget - R, st.status))
+                src[S + dst + __popc(keep_mask & lt)] = S + i;
             dst += __popc(keep_mask);
             const unsigned gone = __ballot_sync(0xffffffffu, i < seg_e && !keep);
             if (gone != 0u && first_evicted == ncand) first_evicted = i0 + __ffs(gone) - 1;
@@ -264,7 +267,7 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(Geometry ge
     const int u = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int32_t* src = a.src + (size_t)u * a.budget;
     const int32_t* pt_g = st.page_table + (size_t)u * geo.pages_per_unit;
-    const int first = a.first_moved[u];
+    const int first = in_bounds(a.first_moved[u] >= 0, st.status) ? a.first_moved[u] : a.budget;
     const size_t sbase = (size_t)u * geo.capacity;
     const int half = lane < 16 ? 0 : kPageHalfBytes;      // lanes 0..15: K row, 16..31: V row
     const int cp = lane & 15;                             // physical chunk read from the source row
@@ -278,7 +281,14 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(Geometry ge
     auto source_of = [&](int dj) -> int {
         if (dj < first || dj >= a.budget) return -1;
         const int sj = src[dj];
+        if (!in_bounds(sj >= dj && sj < a.n, st.status)) return -1;
         return sj != dj ? sj : -1;
+    };
+    // physical page of logical page `lp` of this unit (checked in the debug build)
+    auto page_of = [&](int lp) -> int32_t {
+        if (!in_bounds(lp >= 0 && lp < geo.pages_per_unit, st.status)) return 0;
+        const int32_t pp = pt[lp];
+        return in_bounds(pp >= 0 && pp < geo.units * geo.pages_per_unit, st.status) ? pp : 0;
     };
 
     int d0 = first / kPageTokens * kPageTokens;
@@ -293,7 +303,7 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(Geometry ge
         for (int i = 0; i < kRowsPerWarp; ++i)
             if (srow[i] >= 0) {
                 const uint8_t* row =
-                    page_ptr(pool, pt[srow[i] / kPageTokens]) + half + (srow[i] % kPageTokens) * kRowBytes;
+                    page_ptr(pool, page_of(srow[i] / kPageTokens)) + half + (srow[i] % kPageTokens) * kRowBytes;
                 val[i] = *reinterpret_cast<const uint4*>(row + cp * 16);
             }
         int s_ts = 0, s_mri = 0, s_pos = 0;
@@ -309,7 +319,7 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(Geometry ge
         if (tid < kPageTokens) s_from_next = source_of(d0 + kPageTokens + tid);
 
         __syncthreads();       // every source row of this tile is in registers
-        uint8_t* dpage = page_ptr(pool, pt[d0 / kPageTokens]) + half;
+        uint8_t* dpage = page_ptr(pool, page_of(d0 / kPageTokens)) + half;
 #pragma unroll
         for (int i = 0; i < kRowsPerWarp; ++i) {
             if (srow[i] >= 0) {

@@ -13,8 +13,8 @@
 // so the heads that share the K / V tile sit in neighbouring lanes.  Every query tile makes
 // two passes over its key tiles (128 keys each):
 //   pass A: S = Q K^T, row maximum and sum of exponentials  ->  exact log-sum-exp per row;
-//   pass B: S = Q K^T again, p = exp2(s - lse) (already normalised), P to shared memory as bf16,
-//           O += P V (no rescaling ever), pbar by a butterfly sum over the GP lanes of a position,
+//   pass B: S = Q K^T again, p = exp2(s - lse) (already normalised), P to shared memory as two bf16
+//           terms (hi + lo), O += P V (no rescaling ever), pbar by a butterfly sum over the GP lanes of a position,
 //           threshold test, activation bits per key column; after the tile one thread per key
 //           column applies Eq. (1) for the tile's positions in ascending order.
 // Key columns are owned by a fixed thread for the whole unit and query tiles are visited in ascending
@@ -41,9 +41,9 @@ constexpr int kPromptThreads = 192;
 constexpr int kOffQ = 0;
 constexpr int kOffKV = kOffQ + kOperandBytes;                       // per stage: K tile, then V tile
 constexpr int kOffP = kOffKV + kKvStages * 2 * kOperandBytes;
-constexpr int kOffMisc = kOffP + kOperandBytes;
+constexpr int kOffMisc = kOffP + 2 * kOperandBytes;                 // P as two bf16 terms: hi tile, lo tile
 constexpr int kMiscBytes = 2048;
-constexpr int kPromptSmem = kOffMisc + kMiscBytes + 1024;           // + slack for the alignment
+constexpr int kPromptSmem = kOffMisc + kMiscBytes;                  // 226 KiB of the 227 KiB a block may have
 
 struct Bars {                                       // mbarriers
     uint64_t q_full, q_empty;
@@ -181,8 +181,7 @@ __global__ void __launch_bounds__(kPromptThreads, 1)
 prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
               const __grid_constant__ CUtensorMap map_v, const PromptParams p) {
     constexpr int TQ = kTile / GP;                  // prompt positions per query tile
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];           // the swizzle atoms need 1024-byte alignment
     uint8_t* q_s = smem + kOffQ;
     uint8_t* p_s = smem + kOffP;
     Bars* bars = reinterpret_cast<Bars*>(smem + kOffMisc);
@@ -325,10 +324,11 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             const uint32_t st = st_of[(kb - 1) & 1];
                             const uint32_t v_addr = smem_u32(smem + kOffKV + st * 2 * kOperandBytes + kOperandBytes);
 #pragma unroll
-                            for (int ks = 0; ks < 8; ++ks) {      // 16 keys per instruction
+                            for (int ks = 0; ks < 8; ++ks) {      // 16 keys per instruction; P = hi + lo, two products
                                 const uint32_t a_off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-                                umma_bf16(tmem_o, smem_desc(p_addr + a_off, 16, 1024),
-                                          smem_desc(v_addr + ks * 2048, kBoxBytes, 1024), idesc_o, (kb > 1 || ks > 0));
+                                const uint64_t v_desc = smem_desc(v_addr + ks * 2048, kBoxBytes, 1024);
+                                umma_bf16(tmem_o, smem_desc(p_addr + a_off, 16, 1024), v_desc, idesc_o, (kb > 1 || ks > 0));
+                                umma_bf16(tmem_o, smem_desc(p_addr + kOperandBytes + a_off, 16, 1024), v_desc, idesc_o, 1u);
                             }
                             umma_commit(&bars->p_empty);
                             umma_commit(&bars->kv_empty[st]);
@@ -414,18 +414,25 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             x[i] = key0 + i <= pos ? fast_exp2(x[i] * p.scale_log2 - lse) : 0.f;
-                        // P as the K-major A operand of O += P V: row `row`, keys key0 .. key0 + 31 of this tile
+                        // P as the K-major A operand of O += P V: row `row`, keys key0 .. key0 + 31 of this tile.
+                        // It enters the tensor core as two bf16 terms, p = hi + lo (16 mantissa bits): with one
+                        // term the weights would be off by up to 2^-9, more than the output tolerance allows
+                        // where large values cancel.
                         {
                             uint8_t* prow = p_s + (c >> 1) * kBoxBytes + row * 128;
 #pragma unroll
                             for (int ch = 0; ch < 4; ++ch) {
-                                uint4 w;
-                                w.x = pack_bf16(x[8 * ch + 0], x[8 * ch + 1]);
-                                w.y = pack_bf16(x[8 * ch + 2], x[8 * ch + 3]);
-                                w.z = pack_bf16(x[8 * ch + 4], x[8 * ch + 5]);
-                                w.w = pack_bf16(x[8 * ch + 6], x[8 * ch + 7]);
+                                uint32_t hi[4], lo[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float a0 = x[8 * ch + 2 * e], a1 = x[8 * ch + 2 * e + 1];
+                                    hi[e] = pack_bf16(a0, a1);
+                                    lo[e] = pack_bf16(a0 - bf16_lo_as_float(hi[e]), a1 - bf16_hi_as_float(hi[e]));
+                                }
                                 const int chunk = (c & 1) * 4 + ch;
-                                *reinterpret_cast<uint4*>(prow + ((chunk ^ (row & 7)) << 4)) = w;
+                                uint8_t* dst = prow + ((chunk ^ (row & 7)) << 4);
+                                *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+                                *reinterpret_cast<uint4*>(dst + kOperandBytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                             }
                         }
                         // pbar: sum over the GP lanes of this position.  Every round halves what a lane keeps,

@@ -458,6 +458,74 @@ def test_step_whose_automatic_eviction_cannot_run_is_refused_up_front():
     assert eng.counters().device_status == 0
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_recovers():
+    """The decode kernel's waits are bounded: a block whose page ring is starved (a diagnostic switch
+    makes the producer warp stop after two pages) gives up after the wait limit, the kernel ends by
+    itself, the status word says so, and after lazyev_reset the handle serves a new sequence with the
+    results of a fresh handle.  Nothing faults and the CUDA context stays usable throughout."""
+    from tests.harness import make_engine
+    cfg = traces.tiny_config(batch=1, layers=1, prefill=300, budget=400)          # 2 units, 5 pages each
+    shape = (cfg.layers, cfg.batch, cfg.kv_heads, cfg.prefill, 128)
+    used, fresh = make_engine(cfg), make_engine(cfg)
+    used.set_splits(1); fresh.set_splits(1)
+    used.set_wait_limit(0.004)
+    out_u = torch.empty(cfg.layers, cfg.batch, cfg.q_heads, 128, dtype=torch.bfloat16, device="cuda")
+    out_f = torch.empty_like(out_u)
+    gen = traces.TraceGen(cfg, 40, device="cuda")
+    k, v = gen.prefill()
+    used.prefill(k.view(shape), v.view(shape))
+    q, kn, vn = gen.steps(4)
+    used.decode_step(q[0], kn[0], vn[0], out_u)
+    used.synchronize()                                        # a healthy step first
+    used.debug_starve_page_ring(2)
+    used.decode_step(q[1], kn[1], vn[1], out_u)               # queued; the kernel gives up after ~4 ms
+    with pytest.raises(binding.LazyEvError) as e:
+        used.synchronize()
+    assert e.value.code == binding.EDEVICE
+    assert used.counters().device_status & 1                  # "a bounded wait gave up"
+    torch.cuda.synchronize()                                  # the context is alive
+    used.debug_starve_page_ring(-1)
+    used.reset()
+    assert used.counters().device_status == 0
+    gen2 = traces.TraceGen(cfg, 41, device="cuda")
+    k, v = gen2.prefill()
+    used.prefill(k.view(shape), v.view(shape)); fresh.prefill(k.view(shape), v.view(shape))
+    for _ in range(4):                                        # 128 steps with evictions
+        q, kn, vn = gen2.steps(32)
+        for s in range(32):
+            used.decode_step(q[s], kn[s], vn[s], out_u)
+            fresh.decode_step(q[s], kn[s], vn[s], out_f)
+            assert torch.equal(out_u, out_f)
+    du, df = used.dump_state(kv=True), fresh.dump_state(kv=True)
+    for key in ("pos", "ts", "mri", "pbar", "k", "v"):
+        assert np.array_equal(du[key], df[key]), key
+    assert du["device_status"] == 0 and used.info().evictions == fresh.info().evictions + 0
+
+
+def test_library_flavour_is_the_one_the_environment_asks_for():
+    assert bool(binding.lib().lazyev_build_flags() & 1) == binding.debug_bounds_requested()
+
+
+def test_range_checked_build_runs_the_lockstep_tests_clean():
+    """The sanitizer substitute: the same sources compiled with every slot, page-table and work-list
+    index range-checked (a failed check flags the device status word).  The lock-step tests, the
+    random-shape sweep and the prompt tests run again through that build in a child process; they
+    assert a clean status word themselves."""
+    import os, subprocess, sys
+    if binding.debug_bounds_requested():
+        pytest.skip("already inside the range-checked run")
+    env = dict(os.environ, LAZYEV_DEBUG_BOUNDS="1")
+    here = os.path.dirname(os.path.abspath(__file__))
+    sel = ("lockstep_with_evictions or random_shapes or many_units or group_sizes or observed_prompt or "
+           "partly_filled or protected_tokens or dynamic_budget or window_of_one or library_flavour or "
+           "long_contexts or histogram")
+    res = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_parity.py"),
+                          os.path.join(here, "test_zz_no_alloc.py"), "-q", "-x", "-m", "gpu", "-k",
+                          sel + " or static_scratch"], env=env, capture_output=True, text=True, cwd=os.path.dirname(here))
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-2000:]
+    assert " passed" in res.stdout and "failed" not in res.stdout
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     cfg = traces.tiny_config()
     gen = traces.TraceGen(cfg, 8, device="cuda")
