@@ -273,7 +273,7 @@ int lazyev_evict(lazyev_t* h, int* evicted);
  * This entry point does exactly what lazyev_evict() does -- same trigger test, same kernels,
  * same results bit for bit, same profiling records -- but keeps the source lists and
  * first-moved indices (the part of the scratch region that grows with units * budget) in an
- * array that is compiled into the library (4 MiB + 16 KiB of device memory on every GPU that
+ * array that is compiled into the library (4 MiB + 32 KiB of device memory on every GPU that
  * loads the library, held until the process exits).  It calls no device allocator of any kind.
  * lazyev_bind() still wants a scratch region of the size lazyev_query_sizes() reports (the
  * staging buffers and the 256 KiB table of H2 terms live there); a caller that only ever uses

@@ -38,6 +38,7 @@ struct lazyev {
     StateView st = {};
     int32_t* src = nullptr;
     int32_t* first_moved = nullptr;
+    int32_t* radix_list = nullptr;         // [units] + the counter behind it
     // staging of the host-buffer entry points: two slots, so that the copies of one step run beside
     // the kernels of the step before it
     uint8_t* stage_q[2] = {nullptr, nullptr};
@@ -114,7 +115,7 @@ void derive(lazyev_t* h) {
 struct Sizes {
     size_t kv, state, scratch;
     size_t off_ts, off_mri, off_pos, off_pbar, off_status;                          // inside state
-    size_t off_first, off_q, off_k, off_v, off_out, off_score, off_hist, off_h2;    // inside scratch
+    size_t off_first, off_rlist, off_q, off_k, off_v, off_out, off_score, off_hist, off_h2;    // inside scratch
 };
 
 Sizes sizes_of(const lazyev_t* h) {
@@ -136,6 +137,8 @@ Sizes sizes_of(const lazyev_t* h) {
     off = align_up((size_t)h->units * h->budget * sizeof(int32_t), 256);
     s.off_first = off;
     off += align_up((size_t)h->units * sizeof(int32_t), 256);
+    s.off_rlist = off;
+    off += align_up(((size_t)h->units + 1) * sizeof(int32_t), 256);
     const size_t qbytes = (size_t)h->layers * h->batch * h->q_heads * kRowBytes;
     const size_t kbytes = (size_t)h->layers * h->batch * h->kv_heads * kRowBytes;
     s.off_q = off;                          // each staging area holds two slots
@@ -231,7 +234,7 @@ bool evict_due_at(const lazyev_t* h, int t, int n) { return t != 0 && t % h->win
 
 // The lagged eviction of Section 4 at the current step, if one is due.  `src` and `first_moved` are
 // the work lists of the select and compact kernels: the bound scratch region's or the library's own.
-int run_evict(lazyev_t* h, int* evicted, int32_t* src, int32_t* first_moved) {
+int run_evict(lazyev_t* h, int* evicted, int32_t* src, int32_t* first_moved, int32_t* radix_list) {
     if (evicted) *evicted = 0;
     if (!evict_due_at(h, h->t, h->n)) return LAZYEV_OK;
     const int ncand = candidates_of(h, h->n);
@@ -255,13 +258,16 @@ int run_evict(lazyev_t* h, int* evicted, int32_t* src, int32_t* first_moved) {
     a.first_moved = first_moved;
     a.h2_table = h->h2_table;
     a.h2_entries = kH2TableEntries;
+    a.radix_list = radix_list;
+    a.radix_count = radix_list + h->units;
     const Geometry geo = geometry(h);
     {
         // algorithmic bytes: TS and MRI of every candidate read, the source list written
         SpanGuard g(h, kSpanSelect, (double)h->units * (8.0 * ncand + 4.0 * a.budget));
-        e = select_launch(geo, h->st, a, h->stream);
+        e = select_launch(geo, h->st, a, h->num_sms, h->stream);
     }
     if (e != cudaSuccess) return cuda_fail(h, e, "select kernel launch");
+    h->launches += 1;        // the selection is two launches
     {
         SpanGuard g(h, kSpanCompact, 0.0);
         e = compact_launch(geo, h->pool, h->st, a, h->stream);
@@ -476,7 +482,7 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
     if (rc != LAZYEV_OK) return rc;
     h->t = t;
     h->n = n;
-    if (h->auto_evict) return run_evict(h, nullptr, h->src, h->first_moved);
+    if (h->auto_evict) return run_evict(h, nullptr, h->src, h->first_moved, h->radix_list);
     return LAZYEV_OK;
 }
 
@@ -633,6 +639,7 @@ int lazyev_bind(lazyev_t* h, void* kv_pool, void* state, void* scratch, void* cu
     uint8_t* cp = (uint8_t*)scratch;
     h->src = (int32_t*)cp;
     h->first_moved = (int32_t*)(cp + s.off_first);
+    h->radix_list = (int32_t*)(cp + s.off_rlist);
     {
         const size_t qslot = align_up((size_t)h->layers * h->batch * h->q_heads * kRowBytes, 256);
         const size_t kslot = align_up((size_t)h->layers * h->batch * h->kv_heads * kRowBytes, 256);
@@ -932,16 +939,17 @@ int lazyev_copy_state(lazyev_t* dst, lazyev_t* src) {
 int lazyev_evict(lazyev_t* h, int* evicted) {
     if (!h) return LAZYEV_EINVAL;
     if (!h->prefilled) return fail(h, LAZYEV_ESTATE, "evict before prefill");
-    return run_evict(h, evicted, h->src, h->first_moved);
+    return run_evict(h, evicted, h->src, h->first_moved, h->radix_list);
 }
 
 // ---- eviction without caller-provided scratch ------------------------------------------------
 // Source lists and first-moved indices of lazyev_evict_static(): one array per GPU that loads the
-// library, held until the process exits.  4 MiB + 16 KiB.
+// library, held until the process exits.  4 MiB + 32 KiB: source lists, first-moved indices, and the list
+// of units that take the selection's general route.
 constexpr size_t kStaticSrcEntries = (size_t)1 << 20;      // units * budget_now must not exceed this
 constexpr int kStaticMaxUnits = 4096;
 constexpr int kStaticMaxDevices = 64;
-static __device__ __align__(256) int32_t g_static_evict_scratch[kStaticSrcEntries + kStaticMaxUnits];
+static __device__ __align__(256) int32_t g_static_evict_scratch[kStaticSrcEntries + 2 * kStaticMaxUnits + 64];
 // Device addresses of the array above, one per device ordinal.  The symbol itself is only a
 // host-side stand-in: kernels must be given the address cudaGetSymbolAddress() returns.
 static std::atomic<int32_t*> g_static_evict_ptr[kStaticMaxDevices];
@@ -970,7 +978,7 @@ int lazyev_evict_static(lazyev_t* h, int* evicted) {
     // Same trigger test, kernels, timing spans and accounting as lazyev_evict(); only the work lists
     // live elsewhere.  Every entry below budget is rewritten by the select kernel before the compact
     // kernel reads it, so nothing in the array has to be cleared.
-    return run_evict(h, evicted, base, base + kStaticSrcEntries);
+    return run_evict(h, evicted, base, base + kStaticSrcEntries, base + kStaticSrcEntries + kStaticMaxUnits);
 }
 
 int lazyev_get_counters(lazyev_t* h, lazyev_counters_t* out) {

@@ -355,6 +355,17 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         };
         if (my_units > 0) load_q(p.unit_begin + cluster_id, qb);
 
+        // Pages belong to the groups in turn (page pc of the block's walk to group pc mod NG, across unit
+        // boundaries), and a warp looks at the barriers up to its own next page before it releases the
+        // page it holds; the producer refills a stage only after the pages before it were released, so it
+        // cannot lap a barrier that some warp has not looked at -- provided every warp has looked at the
+        // first NG pages before the first release.  With fewer pages per unit than groups a group's first
+        // page lies behind the first unit's merge, so that is made sure of here, once.
+        if (NG > 1) {
+            observe_through((uint32_t)(NG - 1));
+            named_barrier_sync(1, kConsumers);
+        }
+
         for (int u = p.unit_begin + cluster_id; u < p.unit_end; u += n_clusters, ++it) {
             uint32_t qn[8][2] = {};
             if (u + n_clusters < p.unit_end) load_q(u + n_clusters, qn);

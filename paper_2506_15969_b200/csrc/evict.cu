@@ -1,8 +1,10 @@
 // Lagged eviction (Section 4 "MRI-Centric Eviction" of the paper):
 //   score_fn       -- H1, H2 and Eq. (2), fp64
-//   select_kernel  -- top-(B - R - S) of the unprotected slots by (score, recency): block-wide radix
-//                     select on the fp64 score bits, then a prefix sum that turns keep flags into the
-//                     list "slot src[j] moves to slot j" (Appendix A, Eq. (evic))
+//   select_fast_kernel -- top-(B - R - S) of the unprotected slots by (score, recency) when the k-th
+//                     score is 0 (only zero / non-zero matters, no floating point), else lists the unit
+//   select_kernel  -- the general route for listed units: fp64 scores, block-wide radix select on the
+//                     score bits, then a prefix sum that turns keep flags into the list "slot src[j]
+//                     moves to slot j" (Appendix A, Eq. (evic))
 //   compact_kernel -- in-place, order-preserving gather of K, V, TS, MRI and positions (Algorithm 1,
 //                     "update KV pairs")
 #include "internal.h"
@@ -72,14 +74,22 @@ __device__ __forceinline__ int block_sum(int v, int* warp_sums) {
     return s;
 }
 
-__global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, StateView st, EvictArgs a) {
-    extern __shared__ __align__(16) unsigned long long keys[];
-    __shared__ unsigned int hist[256];
-    __shared__ unsigned long long sh_prefix;
-    __shared__ int sh_krem, sh_first, sh_done;
-    __shared__ int warp_sums[kSelThreads / 32];
+struct SelectShared {
+    unsigned int hist[256];
+    unsigned long long prefix;
+    int krem, first, done;
+    int warp_sums[kSelThreads / 32];
+};
 
-    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+// The selection of one unit with the k-th score found by radix passes (the general route).
+__device__ void select_radix_unit(const int u, const Geometry& geo, const StateView& st, const EvictArgs& a,
+                                  unsigned long long* keys, SelectShared& sh) {
+    unsigned int* hist = sh.hist;
+    unsigned long long& sh_prefix = sh.prefix;
+    int &sh_krem = sh.krem, &sh_first = sh.first, &sh_done = sh.done;
+    int* warp_sums = sh.warp_sums;
+
+    const int tid = threadIdx.x, lane = tid & 31;
     const int S = a.n_initial, R = a.n_recent;
     const int ncand = a.n - R - S;                 // unprotected slots [S, n - R)
     const int k = a.budget - R - S;                // how many of them stay
@@ -127,7 +137,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     // kth: bit pattern of the k-th largest score; krem: how many of the keys equal to it stay.
     unsigned long long kth = 0;
     int krem = k - nonzero;
-    if (tid == 0) atomicAdd(st.status + (nonzero > k ? kCounterRadixUnits : kCounterZeroCutUnits), 1);
     if (nonzero > k) {
         // More non-zero scores than tokens to keep: the k-th score has to be found.  Eq. (2) in fp64 for
         // every non-zero candidate (most of them in this regime, so the warps stay converged) ...
@@ -245,6 +254,153 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, State
     for (int j = tid; j < S; j += kSelThreads) src[j] = j;
     for (int r = tid; r < R; r += kSelThreads) src[a.budget - R + r] = a.n - R + r;
     __syncthreads();
+    if (tid == 0) {
+        a.first_moved[u] = S + sh_first;
+        if (total_kept != k) atomicOr(st.status, kStatusBadIndex);
+    }
+}
+
+// Blocks take the units that select_fast_kernel listed for the general route.
+__global__ void __launch_bounds__(kSelThreads) select_kernel(Geometry geo, StateView st, EvictArgs a) {
+    extern __shared__ __align__(16) unsigned long long keys[];
+    __shared__ SelectShared sh;
+    const int listed = *a.radix_count;
+    for (int idx = blockIdx.x; idx < listed; idx += gridDim.x) {
+        select_radix_unit(a.radix_list[idx], geo, st, a, keys, sh);
+        __syncthreads();
+    }
+}
+
+constexpr int kMaxSelSteps = 64;       // 32 candidates per step and warp: up to 32768 candidates per unit
+
+// First stage of the selection, for every unit: classify every candidate's score as zero or not (no
+// floating point, see select_radix_unit) into one bit per candidate.  If at most k scores are non-zero
+// -- the usual case: the tokens an eviction removes are the ones never re-activated -- the k-th score is
+// 0, every non-zero score stays, and of the zeros the most recent stay (the tie rule): the keep flags,
+// their ranks and the source list all follow from the bit words, and the unit is done.  Otherwise the
+// unit is put on the list for select_kernel.
+__global__ void __launch_bounds__(kSelThreads) select_fast_kernel(Geometry geo, StateView st, EvictArgs a) {
+    constexpr int kWarps = kSelThreads / 32;
+    __shared__ uint32_t nzw[kWarps][kMaxSelSteps];      // bit = this candidate's score is not zero
+    __shared__ uint32_t keepw[kWarps][kMaxSelSteps];    // bit = this candidate stays
+    __shared__ int dbase[kWarps][kMaxSelSteps];         // kept candidates of the warp before this word
+    __shared__ int warp_nz[kWarps], warp_kept[kWarps];
+    __shared__ int sh_first;
+
+    const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int S = a.n_initial, R = a.n_recent;
+    const int ncand = a.n - R - S, k = a.budget - R - S;
+    const int32_t* ts = st.ts + (size_t)u * geo.capacity + S;
+    const int32_t* mri = st.mri + (size_t)u * geo.capacity + S;
+    int32_t* src = a.src + (size_t)u * a.budget;
+    if (!in_bounds(S >= 0 && R >= 0 && ncand > 0 && k >= 0 && k <= ncand && a.n <= geo.capacity && a.budget <= a.n, st.status))
+        return;
+    const int seg = ((ncand + kWarps - 1) / kWarps + 31) / 32 * 32;
+    const int seg_b = min(ncand, warp * seg), seg_e = min(ncand, seg_b + seg);
+    const int nsteps = (seg_e - seg_b + 31) / 32;
+    const unsigned lt = (1u << lane) - 1u;
+
+    int nz_warp = 0;
+    for (int step = 0; step < nsteps; ++step) {
+        const int i = seg_b + step * 32 + lane;
+        bool nz = false;
+        if (i < seg_e) {
+            const int m = mri[i], d = a.t - ts[i];
+            if (a.score_mode == 2)
+                nz = m > 1;
+            else if (m == 0)
+                nz = d == 0;
+            else if ((long long)d > 700ll * m)
+                nz = score_with_table(d, m, a.score_mode, a.h2_table, a.h2_entries) != 0.0;
+            else
+                nz = true;
+        }
+        const unsigned word = __ballot_sync(0xffffffffu, nz);
+        if (lane == 0) nzw[warp][step] = word;
+        nz_warp += __popc(word);
+    }
+    if (lane == 0) warp_nz[warp] = nz_warp;
+    if (tid == 0) sh_first = ncand;
+    __syncthreads();
+    int nonzero = 0, zeros_before = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        nonzero += warp_nz[w];
+        const int wb = min(ncand, w * seg), we = min(ncand, wb + seg);
+        zeros_before += w < warp ? (we - wb) - warp_nz[w] : 0;
+    }
+    if (nonzero > k) {                             // the k-th score is not zero: the general route
+        if (tid == 0) {
+            a.radix_list[atomicAdd(a.radix_count, 1)] = u;
+            atomicAdd(st.status + kCounterRadixUnits, 1);
+        }
+        return;
+    }
+    if (tid == 0) atomicAdd(st.status + kCounterZeroCutUnits, 1);
+
+    // Of the zeros, the first `drop_total` in slot order go (ties are resolved towards the more recent
+    // token); lane l of a warp handles the warp's words l and l + 32.
+    const int drop_total = (ncand - nonzero) - (k - nonzero);
+    int tie_carry = zeros_before, kept_carry = 0, first_gone = ncand;
+    for (int c = 0; c * 32 < nsteps; ++c) {
+        const int step = c * 32 + lane;
+        const bool valid = step < nsteps;
+        const int left = valid ? min(32, seg_e - (seg_b + step * 32)) : 0;
+        const unsigned in_mask = left >= 32 ? 0xffffffffu : ((1u << left) - 1u);
+        const unsigned nz = valid ? nzw[warp][step] : 0u;
+        const unsigned z = ~nz & in_mask;
+        const int cz = __popc(z), ck_nz = __popc(nz);
+        int incl = cz;                             // zeros of this warp up to and including this word
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const int rank0 = tie_carry + incl - cz;   // rank among all zeros of this word's first zero
+        const int drop = min(max(drop_total - rank0, 0), cz);
+        unsigned zk = z;
+        if (drop >= cz)
+            zk = 0u;
+        else
+            for (int q = 0; q < drop; ++q) zk &= zk - 1u;      // clears the lowest set bit
+        const unsigned kw = nz | zk;
+        const int ck = ck_nz + __popc(zk);
+        int inclk = ck;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, inclk, o);
+            if (lane >= o) inclk += up;
+        }
+        if (valid) {
+            keepw[warp][step] = kw;
+            dbase[warp][step] = kept_carry + inclk - ck;
+            const unsigned gone = in_mask & ~kw;
+            if (gone != 0u) first_gone = min(first_gone, seg_b + step * 32 + __ffs(gone) - 1);
+        }
+        tie_carry += __shfl_sync(0xffffffffu, incl, 31);
+        kept_carry += __shfl_sync(0xffffffffu, inclk, 31);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) first_gone = min(first_gone, __shfl_xor_sync(0xffffffffu, first_gone, o));
+    if (lane == 0) {
+        warp_kept[warp] = kept_carry;
+        if (first_gone < ncand) atomicMin(&sh_first, first_gone);
+    }
+    __syncthreads();
+    int warp_dst = 0, total_kept = 0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) {
+        warp_dst += w < warp ? warp_kept[w] : 0;
+        total_kept += warp_kept[w];
+    }
+    // source list: kept candidate number j of the unit moves to slot S + j
+    for (int step = 0; step < nsteps; ++step) {
+        const unsigned kw = keepw[warp][step];
+        const int j = warp_dst + dbase[warp][step] + __popc(kw & lt);
+        if (((kw >> lane) & 1u) && in_bounds(j < k, st.status)) src[S + j] = S + seg_b + step * 32 + lane;
+    }
+    for (int j = tid; j < S; j += kSelThreads) src[j] = j;
+    for (int r = tid; r < R; r += kSelThreads) src[a.budget - R + r] = a.n - R + r;
     if (tid == 0) {
         a.first_moved[u] = S + sh_first;
         if (total_kept != k) atomicOr(st.status, kStatusBadIndex);
@@ -392,9 +548,22 @@ cudaError_t select_prepare() {
     return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
 }
 
-cudaError_t select_launch(const Geometry& geo, StateView st, const EvictArgs& a, cudaStream_t stream) {
+cudaError_t select_launch(const Geometry& geo, StateView st, const EvictArgs& a, int num_sms, cudaStream_t stream) {
     const int ncand = a.n - a.n_recent - a.n_initial;
-    select_kernel<<<geo.units, kSelThreads, select_smem_bytes(ncand), stream>>>(geo, st, a);
+    if (ncand > 32 * kMaxSelSteps * (kSelThreads / 32)) return cudaErrorInvalidValue;
+    cudaError_t e = cudaMemsetAsync(a.radix_count, 0, sizeof(int32_t), stream);
+    if (e != cudaSuccess) return e;
+    select_fast_kernel<<<geo.units, kSelThreads, 0, stream>>>(geo, st, a);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    // the general route for the units the first stage listed: a grid that fills the GPU once
+    const size_t smem = select_smem_bytes(ncand);
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, select_kernel, kSelThreads, smem) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        per_sm = 1;
+    }
+    const int blocks = geo.units < num_sms * per_sm ? geo.units : num_sms * per_sm;
+    select_kernel<<<blocks, kSelThreads, smem, stream>>>(geo, st, a);
     return cudaGetLastError();
 }
 

@@ -74,6 +74,8 @@ struct EvictArgs {
     int32_t* first_moved;  // [units]: first j with src[j] != j (budget if none)
     const double* h2_table;   // H2 term of the score per MRI value, for the mode in score_mode
     int h2_entries;
+    int32_t* radix_list;   // [units]: units whose k-th score is not zero (filled by the first select stage)
+    int32_t* radix_count;  // [1]
 };
 
 constexpr int kH2TableEntries = 1 << 15;    // MRI values covered by the table; larger ones are evaluated directly
@@ -82,7 +84,7 @@ cudaError_t h2_table_launch(int score_mode, int entries, double* table, cudaStre
 
 size_t select_smem_bytes(int n_candidates);
 cudaError_t select_prepare();
-cudaError_t select_launch(const Geometry& geo, StateView st, const EvictArgs& a, cudaStream_t stream);
+cudaError_t select_launch(const Geometry& geo, StateView st, const EvictArgs& a, int num_sms, cudaStream_t stream);
 cudaError_t compact_launch(const Geometry& geo, uint8_t* pool, StateView st, const EvictArgs& a,
                            cudaStream_t stream);
 // Eq. (2) for every slot < n of units [unit_begin, unit_begin + unit_count) into out[unit][capacity].

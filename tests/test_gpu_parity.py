@@ -99,6 +99,19 @@ def test_many_units_per_block(groups):
     assert ls.rep.evictions == 2
 
 
+@pytest.mark.parametrize("groups", [1, 2])
+def test_many_units_with_fewer_pages_than_warp_groups(groups):
+    """Thousands of units with one or two pages each: every block walks two dozen units, a group of
+    consumer warps owns no page in every other unit, and the page ring is reused many times (the
+    order in which warps look at the ring's barriers must hold across unit boundaries)."""
+    cfg = traces.tiny_config(batch=32, layers=28, q_heads=8, kv_heads=4, budget=200, window=32, prefill=10)
+    assert cfg.units == 3584
+    ls = lockstep(cfg, seed=19, sample_units=[0, 147, 148, 2000, 3551, 3552, 3583], groups=groups, pure=False)
+    ls.run(70)                                                # 11 .. 80 cached tokens: crosses the one-page boundary
+    ls.assert_ok()
+    assert ls.eng.counters().device_status == 0
+
+
 @pytest.mark.parametrize("q_heads,kv_heads", [(7, 1), (10, 2), (8, 1), (2, 2), (6, 2)])
 def test_group_sizes(q_heads, kv_heads):
     cfg = traces.tiny_config(q_heads=q_heads, kv_heads=kv_heads, batch=3, layers=1, budget=400, prefill=70)
