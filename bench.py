@@ -40,9 +40,9 @@ FALLBACK_HBM_GBS = 6650.0
 # units x tokens, so a full launch is scaled by its algorithmic bytes.  Valid only for the kernel
 # sources it was taken on.
 NCU_DECODE_CAPTURE = {
-    "traffic_per_algorithmic_byte": 1.0075,
-    "sha256": {"decode.cu": "a4ecc7346b7141d70069dd3e73dafa326a2d20008d509c194be4842d22ef22ba",
-               "common.cuh": "e145966ccf290b94a07f9b5374ce552520833824b6b9440fc6aa85adf416adac"},
+    "traffic_per_algorithmic_byte": 1.0076,
+    "sha256": {"decode.cu": "d739e597f7047acf3fdc725e9f668ebab9c5300f20f42208c6054b7e068ba0c8",
+               "common.cuh": "bd1929d12b75ef1f2ea3bd900d3f93f7a39494c3ab52ff7dd9fe31945b995fd2"},
 }
 
 

@@ -300,12 +300,22 @@ __global__ void __launch_bounds__(kSelThreads) select_fast_kernel(Geometry geo, 
     const int nsteps = (seg_e - seg_b + 31) / 32;
     const unsigned lt = (1u << lane) - 1u;
 
+    // (eight steps at a time: all sixteen loads of a lane are in flight before the first ballot, which
+    // is what keeps this pass bound by bandwidth and not by one memory latency per step)
     int nz_warp = 0;
-    for (int step = 0; step < nsteps; ++step) {
-        const int i = seg_b + step * 32 + lane;
-        bool nz = false;
-        if (i < seg_e) {
-            const int m = mri[i], d = a.t - ts[i];
+    for (int s0 = 0; s0 < nsteps; s0 += 8) {
+        int mm[8], tt[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = seg_b + (s0 + q) * 32 + lane;
+            const bool in = s0 + q < nsteps && i < seg_e;
+            mm[q] = in ? __ldg(mri + i) : 0;
+            tt[q] = in ? __ldg(ts + i) : a.t - 1;      // outside: MRI = 0, elapsed 1 -> a zero score
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int m = mm[q], d = a.t - tt[q];
+            bool nz;
             if (a.score_mode == 2)
                 nz = m > 1;
             else if (m == 0)
@@ -314,10 +324,10 @@ __global__ void __launch_bounds__(kSelThreads) select_fast_kernel(Geometry geo, 
                 nz = score_with_table(d, m, a.score_mode, a.h2_table, a.h2_entries) != 0.0;
             else
                 nz = true;
+            const unsigned word = __ballot_sync(0xffffffffu, nz);
+            if (lane == 0 && s0 + q < nsteps) nzw[warp][s0 + q] = word;
+            nz_warp += __popc(word);
         }
-        const unsigned word = __ballot_sync(0xffffffffu, nz);
-        if (lane == 0) nzw[warp][step] = word;
-        nz_warp += __popc(word);
     }
     if (lane == 0) warp_nz[warp] = nz_warp;
     if (tid == 0) sh_first = ncand;

@@ -20,8 +20,9 @@
 // Key columns are owned by a fixed thread for the whole unit and query tiles are visited in ascending
 // order, so every token sees its activations in row order.
 //
-// Warp roles: warps 0-3 softmax / tracking / epilogue (thread = accumulator row = TMEM lane),
-// warp 4 TMA producer, warp 5 MMA issuer.  All mbarrier waits are bounded.
+// Warp roles: warps 0-7 softmax / tracking / epilogue (thread = accumulator row = TMEM lane; the two
+// warps that share a lane quarter take one half of a tile's columns each), warp 8 TMA producer,
+// warp 9 MMA issuer.  All mbarrier waits are bounded.
 #include <cuda.h>
 
 #include "internal.h"
@@ -34,8 +35,9 @@ constexpr int kTile = 128;                         // rows of a query tile, keys
 constexpr int kBoxBytes = kTile * 128;             // one TMA box: 128 rows x 64 bf16 (16 KiB)
 constexpr int kOperandBytes = 2 * kBoxBytes;       // a 128 x 128 bf16 operand tile: two boxes (32 KiB)
 constexpr int kKvStages = 2;
-constexpr int kSoftmaxThreads = 128;
-constexpr int kPromptThreads = 192;
+constexpr int kSoftmaxWarps = 8;                   // two per TMEM lane quarter: each takes half of a tile's columns
+constexpr int kSoftmaxThreads = 32 * kSoftmaxWarps;
+constexpr int kPromptThreads = kSoftmaxThreads + 64;
 
 // shared-memory map (offsets from a 1024-byte aligned base)
 constexpr int kOffQ = 0;
@@ -201,12 +203,12 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars->s_full[i], 1);
-            mbar_init(&bars->s_empty[i], 4);
+            mbar_init(&bars->s_empty[i], kSoftmaxWarps);
         }
-        mbar_init(&bars->p_full, 4);
+        mbar_init(&bars->p_full, kSoftmaxWarps);
         mbar_init(&bars->p_empty, 1);
         mbar_init(&bars->o_full, 1);
-        mbar_init(&bars->o_empty, 4);
+        mbar_init(&bars->o_empty, kSoftmaxWarps);
         mbar_init(&bars->drain, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -226,7 +228,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     // key tiles a query tile needs: all keys up to its last position
     auto key_tiles = [&](int qt) { return (min(P, (qt + 1) * TQ) - 1) / kTile + 1; };
 
-    if (warp == 4) {
+    if (warp == kSoftmaxWarps) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             Ring kv;
@@ -266,7 +268,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 if (q_uses > 0) wait_bar(&bars->q_full, (q_uses - 1) & 1u, abort_flag, p.status, limit, false);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kSoftmaxWarps + 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             Ring kv, sb;                            // K/V stage uses, S buffer uses
@@ -347,10 +349,14 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------------ softmax, tracking, epilogue
-        const int row = threadIdx.x;                // accumulator row = TMEM lane
+        // Warps w and w + 4 share TMEM lanes 32 (w % 4) ..: thread = accumulator row, and the two warps of a
+        // row take the lower and the upper 64 columns of every tile.
+        const int row = threadIdx.x & 127;          // accumulator row = TMEM lane
+        const int chalf = threadIdx.x >> 7;         // which half of the columns
         const int jj = row / GP, g = row % GP;
         const bool head_on = g < G;
-        const uint32_t tmem_row = tmem_base + ((uint32_t)(32 * warp) << 16);
+        const uint32_t tmem_row = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
+        const uint32_t tmem_ml = tmem_row + 384;    // spare columns: the two halves of a row exchange (maximum, sum) here
         Ring sb;
         uint32_t p_uses = 0, o_uses = 0, tiles = 0;
         bool ok = true;
@@ -370,7 +376,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     if (!ok) break;
                     tmem_fence_after_sync();
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 2 * chalf; c < 2 * chalf + 2; ++c) {
                         float x[32];
                         tmem_ld32(tmem_row + buf * 128 + c * 32, x);
                         tmem_wait_ld();
@@ -395,6 +401,20 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     if (lane == 0) mbar_arrive(&bars->s_empty[buf]);
                 }
                 if (!ok) break;
+                // the row's other half of the columns: combine the two (maximum, sum) pairs
+                tmem_st4(tmem_ml + 4 * chalf, m, l, 0.f, 0.f);
+                tmem_wait_st();
+                tmem_fence_before_sync();
+                named_barrier_sync(1, kSoftmaxThreads);
+                tmem_fence_after_sync();
+                {
+                    float om, ol, pad0, pad1;
+                    tmem_ld4(tmem_ml + 4 * (chalf ^ 1), om, ol, pad0, pad1);
+                    tmem_wait_ld();
+                    const float mm = fmaxf(m, om);
+                    l = (m > -INFINITY ? l * fast_exp2(m - mm) : 0.f) + (om > -INFINITY ? ol * fast_exp2(om - mm) : 0.f);
+                    m = mm;
+                }
                 const float lse = m + log2f(l);
                 // ---- pass B: normalised probabilities, P for the tensor core, pbar, activations ----
                 for (int kb = 0; kb < nkb && ok; ++kb, ++sb.count, ++tiles) {
@@ -406,7 +426,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     tmem_fence_after_sync();
                     uint32_t* act_t = act + (tiles & 1u) * kTile;
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 2 * chalf; c < 2 * chalf + 2; ++c) {
                         float x[32];
                         tmem_ld32(tmem_row + buf * 128 + c * 32, x);
                         tmem_wait_ld();
@@ -477,7 +497,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     ++p_uses;
                     // Eq. (1) for this tile's activations: thread `row` owns key column kb * 128 + row.
                     named_barrier_sync(1, kSoftmaxThreads);
-                    const uint32_t bits = act_t[row];
+                    const uint32_t bits = chalf == 0 ? act_t[row] : 0u;
                     if (bits != 0u) {
                         act_t[row] = 0u;
                         const size_t s = srow + (size_t)kb * kTile + row;
@@ -500,7 +520,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                 if (!ok) break;
                 tmem_fence_after_sync();
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 2 * chalf; c < 2 * chalf + 2; ++c) {
                     float x[32];
                     tmem_ld32(tmem_row + 256 + c * 32, x);
                     tmem_wait_ld();
