@@ -7,22 +7,29 @@
 //   pbar[j][i] >= alpha  =>  MRI[i] = max(MRI[i], time_j - TS[i]);  TS[i] = time_j,   time_j = j - (P - 1).
 //
 // This is the one dense contraction of the path, so it runs on the fifth-generation tensor cores:
-// tcgen05.mma with both operands in shared memory (TMA tiles, 128-byte swizzle) and accumulators in
-// tensor memory.  One block owns a unit and walks its query tiles in row order; a query tile is 128
-// rows = (128 / GP) prompt positions x GP query-head slots (GP = 4 or 8, the group size rounded up),
-// so the heads that share the K / V tile sit in neighbouring lanes.  Every query tile makes
-// two passes over its key tiles (128 keys each):
+// tcgen05.mma with operands in shared memory (TMA tiles, 128-byte swizzle) or tensor memory and
+// accumulators in tensor memory.  One block owns a unit and walks its query tiles in row order; a query
+// tile is 128 rows = (128 / GP) prompt positions x GP query-head slots (GP = 4 or 8, the group size
+// rounded up), so the heads that share the K / V tile sit in neighbouring lanes.  Every query tile
+// makes two passes over its key tiles (128 keys each):
 //   pass A: S = Q K^T, row maximum and sum of exponentials  ->  exact log-sum-exp per row;
-//   pass B: S = Q K^T again, p = exp2(s - lse) (already normalised), P to shared memory as two bf16
-//           terms (hi + lo), O += P V (no rescaling ever), pbar by a butterfly sum over the GP lanes of a position,
-//           threshold test, activation bits per key column; after the tile one thread per key
-//           column applies Eq. (1) for the tile's positions in ascending order.
+//   pass B: S = Q K^T again, p = exp2(s - lse) (already normalised) written back over S in tensor
+//           memory as two bf16 terms (hi + lo), O += P V with P as the tensor-memory operand (no
+//           rescaling ever, no shared-memory round trip), pbar by a butterfly sum over the GP lanes of
+//           a position, threshold test, activation bits per key column; after the tile one thread per
+//           key column applies Eq. (1) for the tile's positions in ascending order.
 // Key columns are owned by a fixed thread for the whole unit and query tiles are visited in ascending
 // order, so every token sees its activations in row order.
 //
-// Warp roles: warps 0-7 softmax / tracking / epilogue (thread = accumulator row = TMEM lane; the two
-// warps that share a lane quarter take one half of a tile's columns each), warp 8 TMA producer,
-// warp 9 MMA issuer.  All mbarrier waits are bounded.
+// Pipeline: S is double-buffered in tensor memory, so the tensor core computes the logits of key tile
+// kb + 1 (and, in pass B, O += P V of tile kb - 1) while the softmax warps work on tile kb; K tiles come
+// through a three-stage ring, V tiles through a two-stage ring, and the next query tile's Q is fetched
+// while the current one is worked on.  MMAs issued by one thread execute in issue order, which is what
+// orders "O += P V of tile kb" before "S of tile kb + 2" on the same tensor-memory columns.
+//
+// Warp roles: warps 0-15 softmax / tracking / epilogue (thread = accumulator row = TMEM lane; the four
+// warps that share a lane quarter take 32 of a tile's columns each), warp 16 TMA producer,
+// warp 17 MMA issuer.  All mbarrier waits are bounded.
 #include <cuda.h>
 
 #include "internal.h"
@@ -34,24 +41,28 @@ namespace {
 constexpr int kTile = 128;                         // rows of a query tile, keys of a key tile
 constexpr int kBoxBytes = kTile * 128;             // one TMA box: 128 rows x 64 bf16 (16 KiB)
 constexpr int kOperandBytes = 2 * kBoxBytes;       // a 128 x 128 bf16 operand tile: two boxes (32 KiB)
-constexpr int kKvStages = 2;
-constexpr int kSoftmaxWarps = 8;                   // two per TMEM lane quarter: each takes half of a tile's columns
+constexpr int kKStages = 3, kVStages = 2;
+constexpr int kSoftmaxWarps = 16;                  // four per TMEM lane quarter: each takes 32 of a tile's 128 columns
 constexpr int kSoftmaxThreads = 32 * kSoftmaxWarps;
 constexpr int kPromptThreads = kSoftmaxThreads + 64;
 
-// shared-memory map (offsets from a 1024-byte aligned base)
-constexpr int kOffQ = 0;
-constexpr int kOffKV = kOffQ + kOperandBytes;                       // per stage: K tile, then V tile
-constexpr int kOffP = kOffKV + kKvStages * 2 * kOperandBytes;
-constexpr int kOffMisc = kOffP + 2 * kOperandBytes;                 // P as two bf16 terms: hi tile, lo tile
+// shared-memory map (the base is 1024-byte aligned: the swizzle atoms need it)
+constexpr int kOffQ = 0;                                            // two query tiles
+constexpr int kOffK = kOffQ + 2 * kOperandBytes;
+constexpr int kOffV = kOffK + kKStages * kOperandBytes;
+constexpr int kOffMisc = kOffV + kVStages * kOperandBytes;
 constexpr int kMiscBytes = 2048;
 constexpr int kPromptSmem = kOffMisc + kMiscBytes;                  // 226 KiB of the 227 KiB a block may have
 
+// tensor-memory columns: S / P double buffer, O, and a few spare columns for the row statistics
+constexpr uint32_t kColS = 0, kColO = 256, kColStats = 384, kTmemCols = 512;
+
 struct Bars {                                       // mbarriers
-    uint64_t q_full, q_empty;
-    uint64_t kv_full[kKvStages], kv_empty[kKvStages];
+    uint64_t q_full[2], out_ready[2];               // out_ready: the tile's output sits in its Q slot
+    uint64_t k_full[kKStages], k_empty[kKStages];
+    uint64_t v_full[kVStages], v_empty[kVStages];
     uint64_t s_full[2], s_empty[2];
-    uint64_t p_full, p_empty;
+    uint64_t p_full[2];
     uint64_t o_full, o_empty;
     uint64_t drain;
 };
@@ -59,7 +70,6 @@ struct Bars {                                       // mbarriers
 struct PromptParams {
     int units, group, P, capacity;
     float scale_log2, inv_group, alpha;
-    __nv_bfloat16* out;                             // [P][units][group][128]
     int32_t* ts;
     int32_t* mri;
     float* pbar;
@@ -87,6 +97,17 @@ __device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m
         : "memory");
 }
 
+// Tile store shared -> global through a tensor map (rows outside the tensor are dropped).
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int x, int y, int z, int w, const void* smem_src) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(smem_src))
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {     // arrives once the MMAs issued so far are done
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
@@ -99,6 +120,25 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
         "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// The same with A in tensor memory (row i in lane i, two bf16 per 32-bit column, 8 columns per instruction).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+        "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
 }
 
@@ -158,19 +198,6 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
     return true;
 }
 
-// Barrier over `threads` threads that also ANDs a predicate: every thread learns whether all of them
-// passed their waits, so that they leave the loops together.
-__device__ __forceinline__ bool named_barrier_and(int id, int threads, bool pred) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %3, 0;\n\t"
-        "bar.red.and.pred p, %1, %2, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(r)
-        : "r"(id), "r"(threads), "r"((uint32_t)pred)
-        : "memory");
-    return r != 0;
-}
-
 // One use of a barrier pair in a ring: which stage and which parity a counter of uses maps to.
 struct Ring {
     uint32_t count = 0;
@@ -181,32 +208,34 @@ struct Ring {
 template <int GP>
 __global__ void __launch_bounds__(kPromptThreads, 1)
 prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-              const __grid_constant__ CUtensorMap map_v, const PromptParams p) {
+              const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_out,
+              const PromptParams p) {
     constexpr int TQ = kTile / GP;                  // prompt positions per query tile
-    extern __shared__ __align__(1024) uint8_t smem[];           // the swizzle atoms need 1024-byte alignment
-    uint8_t* q_s = smem + kOffQ;
-    uint8_t* p_s = smem + kOffP;
+    extern __shared__ __align__(1024) uint8_t smem[];
     Bars* bars = reinterpret_cast<Bars*>(smem + kOffMisc);
-    uint32_t* act = reinterpret_cast<uint32_t*>(smem + kOffMisc + 256);          // [2][128] activation bits per key column
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffMisc + 256 + 1024);
+    uint32_t* act = reinterpret_cast<uint32_t*>(smem + kOffMisc + 512);          // [2][128] activation bits per key column
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kOffMisc + 512 + 1024);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int P = p.P, G = p.group;
 
     if (threadIdx.x == 0) {
-        mbar_init(&bars->q_full, 1);
-        mbar_init(&bars->q_empty, 1);
-        for (int i = 0; i < kKvStages; ++i) {
-            mbar_init(&bars->kv_full[i], 1);
-            mbar_init(&bars->kv_empty[i], 1);
-        }
         for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars->q_full[i], 1);
+            mbar_init(&bars->out_ready[i], kSoftmaxWarps);
             mbar_init(&bars->s_full[i], 1);
             mbar_init(&bars->s_empty[i], kSoftmaxWarps);
+            mbar_init(&bars->p_full[i], kSoftmaxWarps);
         }
-        mbar_init(&bars->p_full, kSoftmaxWarps);
-        mbar_init(&bars->p_empty, 1);
+        for (int i = 0; i < kKStages; ++i) {
+            mbar_init(&bars->k_full[i], 1);
+            mbar_init(&bars->k_empty[i], 1);
+        }
+        for (int i = 0; i < kVStages; ++i) {
+            mbar_init(&bars->v_full[i], 1);
+            mbar_init(&bars->v_empty[i], 1);
+        }
         mbar_init(&bars->o_full, 1);
         mbar_init(&bars->o_empty, kSoftmaxWarps);
         mbar_init(&bars->drain, 1);
@@ -215,7 +244,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     }
     for (int i = threadIdx.x; i < 256; i += kPromptThreads) act[i] = 0u;
     if (warp == 0) {
-        tmem_alloc(tmem_slot, 512);                 // S double buffer (2 x 128 columns) + O (128 columns)
+        tmem_alloc(tmem_slot, kTmemCols);
         tmem_relinquish_alloc_permit();
     }
     tmem_fence_before_sync();
@@ -231,115 +260,148 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     if (warp == kSoftmaxWarps) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            Ring kv;
-            uint32_t q_uses = 0;
+            Ring kr, vr, qr;                        // uses of the K ring, the V ring and the two Q slots
             bool ok = true;
+            int slot_u[2] = {0, 0}, slot_qt[2] = {0, 0};
+            auto store_out = [&](uint32_t qs) {    // the output tile in slot qs -> out[positions][unit][heads][128]
+                const uint8_t* o_s = smem + kOffQ + qs * kOperandBytes;
+                tma_store_4d(&map_out, 0, 0, slot_u[qs], slot_qt[qs] * TQ, o_s);
+                tma_store_4d(&map_out, 64, 0, slot_u[qs], slot_qt[qs] * TQ, o_s + kBoxBytes);
+                tma_store_commit();
+                tma_store_wait_read();              // the slot may be overwritten from here on
+            };
             for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
-                for (int qt = 0; qt < n_qt && ok; ++qt, ++q_uses) {
-                    ok = wait_bar(&bars->q_empty, (q_uses & 1u) ^ 1u, abort_flag, p.status, limit);
-                    if (!ok) break;
-                    mbar_arrive_expect_tx(&bars->q_full, kOperandBytes);
-                    tma_load_4d(q_s, &map_q, 0, 0, u, qt * TQ, &bars->q_full);
-                    tma_load_4d(q_s + kBoxBytes, &map_q, 64, 0, u, qt * TQ, &bars->q_full);
+                for (int qt = 0; qt < n_qt && ok; ++qt) {
+                    {
+                        // The slot's previous query tile left its attention output there (the softmax warps
+                        // wrote it once the tile's MMAs were done): send it off, then refill the slot.
+                        const uint32_t qs = qr.stage(2);
+                        if (qr.count >= 2) {
+                            ok = wait_bar(&bars->out_ready[qs], qr.parity(2) ^ 1u, abort_flag, p.status, limit);
+                            if (!ok) break;
+                            store_out(qs);
+                        }
+                        slot_u[qs] = u;
+                        slot_qt[qs] = qt;
+                        uint8_t* q_s = smem + kOffQ + qs * kOperandBytes;
+                        mbar_arrive_expect_tx(&bars->q_full[qs], kOperandBytes);
+                        tma_load_4d(q_s, &map_q, 0, 0, u, qt * TQ, &bars->q_full[qs]);
+                        tma_load_4d(q_s + kBoxBytes, &map_q, 64, 0, u, qt * TQ, &bars->q_full[qs]);
+                        ++qr.count;
+                    }
                     const int nkb = key_tiles(qt);
                     for (int pass = 0; pass < 2 && ok; ++pass) {
-                        for (int kb = 0; kb < nkb; ++kb, ++kv.count) {
-                            const uint32_t st = kv.stage(kKvStages);
-                            ok = wait_bar(&bars->kv_empty[st], kv.parity(kKvStages) ^ 1u, abort_flag, p.status, limit);
+                        for (int kb = 0; kb < nkb; ++kb) {
+                            const uint32_t ks = kr.stage(kKStages);
+                            ok = wait_bar(&bars->k_empty[ks], kr.parity(kKStages) ^ 1u, abort_flag, p.status, limit);
                             if (!ok) break;
-                            uint8_t* k_s = smem + kOffKV + st * 2 * kOperandBytes;
-                            mbar_arrive_expect_tx(&bars->kv_full[st], pass == 0 ? kOperandBytes : 2 * kOperandBytes);
-                            tma_load_3d(k_s, &map_k, 0, kb * kTile, u, &bars->kv_full[st]);
-                            tma_load_3d(k_s + kBoxBytes, &map_k, 64, kb * kTile, u, &bars->kv_full[st]);
+                            uint8_t* k_s = smem + kOffK + ks * kOperandBytes;
+                            mbar_arrive_expect_tx(&bars->k_full[ks], kOperandBytes);
+                            tma_load_3d(k_s, &map_k, 0, kb * kTile, u, &bars->k_full[ks]);
+                            tma_load_3d(k_s + kBoxBytes, &map_k, 64, kb * kTile, u, &bars->k_full[ks]);
+                            ++kr.count;
                             if (pass == 1) {
-                                tma_load_3d(k_s + kOperandBytes, &map_v, 0, kb * kTile, u, &bars->kv_full[st]);
-                                tma_load_3d(k_s + kOperandBytes + kBoxBytes, &map_v, 64, kb * kTile, u, &bars->kv_full[st]);
+                                const uint32_t vs = vr.stage(kVStages);
+                                ok = wait_bar(&bars->v_empty[vs], vr.parity(kVStages) ^ 1u, abort_flag, p.status, limit);
+                                if (!ok) break;
+                                uint8_t* v_s = smem + kOffV + vs * kOperandBytes;
+                                mbar_arrive_expect_tx(&bars->v_full[vs], kOperandBytes);
+                                tma_load_3d(v_s, &map_v, 0, kb * kTile, u, &bars->v_full[vs]);
+                                tma_load_3d(v_s + kBoxBytes, &map_v, 64, kb * kTile, u, &bars->v_full[vs]);
+                                ++vr.count;
                             }
                         }
                     }
                 }
             }
+            if (ok) {
+                // the outputs of the last two query tiles
+                const uint32_t pending = qr.count < 2 ? qr.count : 2;
+                for (uint32_t k = qr.count - pending; k < qr.count && ok; ++k) {
+                    ok = wait_bar(&bars->out_ready[k & 1u], (k >> 1) & 1u, abort_flag, p.status, limit);
+                    if (ok) store_out(k & 1u);
+                }
+            }
+            tma_store_wait_all();
             if (!ok) {
-                // Aborted: let the copies already issued land before the block exits.  The loads of the
-                // last kKvStages stage uses and of the last query tile may still be in flight.
-                const uint32_t last = kv.count < (uint32_t)kKvStages ? kv.count : (uint32_t)kKvStages;
-                for (uint32_t k = kv.count - last; k < kv.count; ++k)
-                    wait_bar(&bars->kv_full[k % kKvStages], (k / kKvStages) & 1u, abort_flag, p.status, limit, false);
-                if (q_uses > 0) wait_bar(&bars->q_full, (q_uses - 1) & 1u, abort_flag, p.status, limit, false);
+                // Aborted: let the copies already issued land before the block exits (the last uses of
+                // every stage may still be in flight).
+                auto drain = [&](uint64_t* full, const Ring& r, uint32_t n) {
+                    const uint32_t last = r.count < n ? r.count : n;
+                    for (uint32_t k = r.count - last; k < r.count; ++k)
+                        wait_bar(&full[k % n], (k / n) & 1u, abort_flag, p.status, limit, false);
+                };
+                drain(bars->k_full, kr, kKStages);
+                drain(bars->v_full, vr, kVStages);
+                drain(bars->q_full, qr, 2);
             }
         }
     } else if (warp == kSoftmaxWarps + 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            Ring kv, sb;                            // K/V stage uses, S buffer uses
-            uint32_t q_uses = 0, p_uses = 0, o_uses = 0;
+            Ring kr, vr, qr, sb;                    // K, V, Q uses and S buffer uses
+            uint32_t p_cnt[2] = {0, 0}, o_uses = 0;
             bool ok = true;
             const uint32_t idesc_s = instr_desc(false), idesc_o = instr_desc(true);
-            const uint32_t q_addr = smem_u32(q_s), p_addr = smem_u32(p_s);
-            const uint32_t tmem_o = tmem_base + 256;
-            // S[buffer] = Q K^T for the K tile in stage `st`
-            auto issue_s = [&](uint32_t st, uint32_t buf) {
-                const uint32_t k_addr = smem_u32(smem + kOffKV + st * 2 * kOperandBytes);
+            const uint32_t tmem_o = tmem_base + kColO;
+            uint32_t q_addr = 0;
+            // S[buffer] = Q K^T for the next K tile of the ring; the K stage is free once these MMAs are done
+            auto issue_s = [&]() -> bool {
+                const uint32_t ks = kr.stage(kKStages), buf = sb.stage(2);
+                if (!(wait_bar(&bars->k_full[ks], kr.parity(kKStages), abort_flag, p.status, limit) &&
+                      wait_bar(&bars->s_empty[buf], sb.parity(2) ^ 1u, abort_flag, p.status, limit)))
+                    return false;
+                tmem_fence_after_sync();
+                const uint32_t k_addr = smem_u32(smem + kOffK + ks * kOperandBytes);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {    // 16 head dimensions per instruction: 32 bytes inside a box row
-                    const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-                    umma_bf16(tmem_base + buf * 128, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024),
-                              idesc_s, ks > 0);
+                for (int s8 = 0; s8 < 8; ++s8) {    // 16 head dimensions per instruction: 32 bytes inside a box row
+                    const uint32_t off = (s8 >> 2) * kBoxBytes + (s8 & 3) * 32;
+                    umma_bf16(tmem_base + kColS + buf * 128, smem_desc(q_addr + off, 16, 1024),
+                              smem_desc(k_addr + off, 16, 1024), idesc_s, s8 > 0);
                 }
+                umma_commit(&bars->s_full[buf]);
+                umma_commit(&bars->k_empty[ks]);
+                ++kr.count;
+                ++sb.count;
+                return true;
             };
             for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
-                for (int qt = 0; qt < n_qt && ok; ++qt, ++q_uses) {
+                for (int qt = 0; qt < n_qt && ok; ++qt) {
                     const int nkb = key_tiles(qt);
-                    ok = wait_bar(&bars->q_full, q_uses & 1u, abort_flag, p.status, limit);
+                    const uint32_t qs = qr.stage(2);
+                    ok = wait_bar(&bars->q_full[qs], qr.parity(2), abort_flag, p.status, limit);
+                    q_addr = smem_u32(smem + kOffQ + qs * kOperandBytes);
                     // pass A: logits only
-                    for (int kb = 0; kb < nkb && ok; ++kb, ++kv.count, ++sb.count) {
-                        const uint32_t st = kv.stage(kKvStages), buf = sb.stage(2);
-                        ok = wait_bar(&bars->kv_full[st], kv.parity(kKvStages), abort_flag, p.status, limit) &&
-                             wait_bar(&bars->s_empty[buf], sb.parity(2) ^ 1u, abort_flag, p.status, limit);
+                    for (int kb = 0; kb < nkb && ok; ++kb) ok = issue_s();
+                    if (!ok) break;
+                    // pass B: logits two tiles ahead, O += P V behind the softmax
+                    const uint32_t first_buf = sb.stage(2);         // buffer of this pass's key tile 0
+                    ok = issue_s();
+                    if (ok && nkb > 1) ok = issue_s();
+                    for (int kb = 0; kb < nkb && ok; ++kb) {
+                        const uint32_t buf = (first_buf + kb) & 1u, vs = vr.stage(kVStages);
+                        ok = wait_bar(&bars->p_full[buf], p_cnt[buf] & 1u, abort_flag, p.status, limit) &&
+                             wait_bar(&bars->v_full[vs], vr.parity(kVStages), abort_flag, p.status, limit);
+                        if (ok && kb == 0) ok = wait_bar(&bars->o_empty, (o_uses & 1u) ^ 1u, abort_flag, p.status, limit);
                         if (!ok) break;
                         tmem_fence_after_sync();
-                        issue_s(st, buf);
-                        umma_commit(&bars->s_full[buf]);
-                        umma_commit(&bars->kv_empty[st]);
-                    }
-                    if (!ok) break;
-                    // pass B: logits, then O += P V one key tile behind
-                    ok = wait_bar(&bars->o_empty, (o_uses & 1u) ^ 1u, abort_flag, p.status, limit);
-                    uint32_t st_of[2] = {0, 0};     // stage of the key tile whose P V product is still to be issued
-                    for (int kb = 0; kb <= nkb && ok; ++kb) {
-                        if (kb < nkb) {
-                            const uint32_t st = kv.stage(kKvStages), buf = sb.stage(2);
-                            ok = wait_bar(&bars->kv_full[st], kv.parity(kKvStages), abort_flag, p.status, limit) &&
-                                 wait_bar(&bars->s_empty[buf], sb.parity(2) ^ 1u, abort_flag, p.status, limit);
-                            if (!ok) break;
-                            tmem_fence_after_sync();
-                            issue_s(st, buf);
-                            umma_commit(&bars->s_full[buf]);
-                            st_of[kb & 1] = st;
-                            ++kv.count;
-                            ++sb.count;
-                        }
-                        if (kb > 0) {               // P of key tile kb - 1 is in shared memory
-                            ok = wait_bar(&bars->p_full, p_uses & 1u, abort_flag, p.status, limit);
-                            if (!ok) break;
-                            tmem_fence_after_sync();
-                            const uint32_t st = st_of[(kb - 1) & 1];
-                            const uint32_t v_addr = smem_u32(smem + kOffKV + st * 2 * kOperandBytes + kOperandBytes);
+                        const uint32_t v_addr = smem_u32(smem + kOffV + vs * kOperandBytes);
+                        const uint32_t p_col = tmem_base + kColS + buf * 128;
 #pragma unroll
-                            for (int ks = 0; ks < 8; ++ks) {      // 16 keys per instruction; P = hi + lo, two products
-                                const uint32_t a_off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-                                const uint64_t v_desc = smem_desc(v_addr + ks * 2048, kBoxBytes, 1024);
-                                umma_bf16(tmem_o, smem_desc(p_addr + a_off, 16, 1024), v_desc, idesc_o, (kb > 1 || ks > 0));
-                                umma_bf16(tmem_o, smem_desc(p_addr + kOperandBytes + a_off, 16, 1024), v_desc, idesc_o, 1u);
-                            }
-                            umma_commit(&bars->p_empty);
-                            umma_commit(&bars->kv_empty[st]);
-                            ++p_uses;
+                        for (int s8 = 0; s8 < 8; ++s8) {            // 16 keys per instruction; P = hi + lo, two products
+                            const uint64_t v_desc = smem_desc(v_addr + s8 * 2048, kBoxBytes, 1024);
+                            const uint32_t a_col = p_col + (s8 >> 1) * 32 + (s8 & 1) * 8;
+                            umma_bf16_ts(tmem_o, a_col, v_desc, idesc_o, (kb > 0 || s8 > 0));
+                            umma_bf16_ts(tmem_o, a_col + 16, v_desc, idesc_o, 1u);
                         }
+                        umma_commit(&bars->v_empty[vs]);
+                        ++vr.count;
+                        ++p_cnt[buf];
+                        if (kb + 2 < nkb) ok = issue_s();           // executes after the product above: same columns
                     }
                     if (!ok) break;
                     umma_commit(&bars->o_full);
-                    umma_commit(&bars->q_empty);
+                    ++qr.count;
                     ++o_uses;
                 }
             }
@@ -349,118 +411,127 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------------ softmax, tracking, epilogue
-        // Warps w and w + 4 share TMEM lanes 32 (w % 4) ..: thread = accumulator row, and the two warps of a
-        // row take the lower and the upper 64 columns of every tile.
+        // Warps w, w + 4, w + 8, w + 12 share TMEM lanes 32 (w % 4) ..: thread = accumulator row, and the four
+        // warps of a row take 32 columns of every tile each (sixteen warps, four per scheduler: the work
+        // is a long chain of exponentials, conversions and shuffles, and needs the warps to hide it).
         const int row = threadIdx.x & 127;          // accumulator row = TMEM lane
-        const int chalf = threadIdx.x >> 7;         // which half of the columns
+        const int c = threadIdx.x >> 7;             // which 32 columns of a tile (and of the output)
         const int jj = row / GP, g = row % GP;
         const bool head_on = g < G;
         const uint32_t tmem_row = tmem_base + ((uint32_t)(32 * (warp & 3)) << 16);
-        const uint32_t tmem_ml = tmem_row + 384;    // spare columns: the two halves of a row exchange (maximum, sum) here
-        Ring sb;
-        uint32_t p_uses = 0, o_uses = 0, tiles = 0;
-        bool ok = true;
-        for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+        const uint32_t tmem_ml = tmem_row + kColStats;      // the two halves of a row exchange (maximum, sum) here
+        // A wait that gives up makes this thread "dead": it keeps walking the same loops, so that every
+        // barrier below still gets all its threads, but it waits for nothing any more (once the abort flag
+        // is up no wait blocks) and what it computes no longer means anything.
+        Ring sb, qr;
+        uint32_t o_uses = 0, tiles = 0;
+        bool dead = false;
+        auto wait_on = [&](uint64_t* bar, uint32_t parity) {
+            if (!dead) dead = !wait_bar(bar, parity, abort_flag, p.status, limit);
+        };
+        for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
             const size_t srow = (size_t)u * p.capacity;
             const bool dumping = p.dump != nullptr && u >= p.dump_begin && u < p.dump_begin + p.dump_count;
-            for (int qt = 0; qt < n_qt && ok; ++qt) {
+            for (int qt = 0; qt < n_qt; ++qt, ++qr.count) {
                 const int pos = qt * TQ + jj;
-                const bool row_on = head_on && pos < P;
                 const int nkb = key_tiles(qt);
                 // ---- pass A: exact log-sum-exp of the row (log2 domain) ----
                 float m = -INFINITY, l = 0.f;
-                for (int kb = 0; kb < nkb && ok; ++kb, ++sb.count) {
+                for (int kb = 0; kb < nkb; ++kb, ++sb.count) {
                     const uint32_t buf = sb.stage(2);
-                    ok = named_barrier_and(2, kSoftmaxThreads,
-                                           wait_bar(&bars->s_full[buf], sb.parity(2), abort_flag, p.status, limit));
-                    if (!ok) break;
+                    wait_on(&bars->s_full[buf], sb.parity(2));
                     tmem_fence_after_sync();
-#pragma unroll 1
-                    for (int c = 2 * chalf; c < 2 * chalf + 2; ++c) {
+                    {
                         float x[32];
-                        tmem_ld32(tmem_row + buf * 128 + c * 32, x);
+                        tmem_ld32(tmem_row + kColS + buf * 128 + c * 32, x);
                         tmem_wait_ld();
                         const int key0 = kb * kTile + c * 32;
-                        float cmax = -INFINITY;
+                        if (key0 + 31 > pos) {      // only the tile on the diagonal has keys beyond the row's position
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            x[i] = key0 + i <= pos ? x[i] * p.scale_log2 : -INFINITY;
-                            cmax = fmaxf(cmax, x[i]);
+                            for (int i = 0; i < 32; ++i) x[i] = key0 + i <= pos ? x[i] : -INFINITY;
                         }
+                        float c0 = fmaxf(x[0], x[1]), c1 = fmaxf(x[2], x[3]), c2 = fmaxf(x[4], x[5]), c3 = fmaxf(x[6], x[7]);
+#pragma unroll
+                        for (int i = 8; i < 32; i += 4) {
+                            c0 = fmaxf(c0, x[i]);
+                            c1 = fmaxf(c1, x[i + 1]);
+                            c2 = fmaxf(c2, x[i + 2]);
+                            c3 = fmaxf(c3, x[i + 3]);
+                        }
+                        const float cmax = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)) * p.scale_log2;     // the scale is positive
                         if (cmax > m) {
                             l *= fast_exp2(m - cmax);     // m = -inf only while l = 0
                             m = cmax;
                         }
                         if (m > -INFINITY) {
+                            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) l += fast_exp2(x[i] - m);
+                            for (int i = 0; i < 32; i += 4) {
+                                l0 += fast_exp2(fmaf(x[i], p.scale_log2, -m));
+                                l1 += fast_exp2(fmaf(x[i + 1], p.scale_log2, -m));
+                                l2 += fast_exp2(fmaf(x[i + 2], p.scale_log2, -m));
+                                l3 += fast_exp2(fmaf(x[i + 3], p.scale_log2, -m));
+                            }
+                            l += (l0 + l1) + (l2 + l3);
                         }
                     }
                     tmem_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&bars->s_empty[buf]);
                 }
-                if (!ok) break;
-                // the row's other half of the columns: combine the two (maximum, sum) pairs
-                tmem_st4(tmem_ml + 4 * chalf, m, l, 0.f, 0.f);
+                // the other parts of the row's columns: combine the four (maximum, sum) pairs
+                tmem_st4(tmem_ml + 4 * c, m, l, 0.f, 0.f);
                 tmem_wait_st();
                 tmem_fence_before_sync();
                 named_barrier_sync(1, kSoftmaxThreads);
                 tmem_fence_after_sync();
                 {
-                    float om, ol, pad0, pad1;
-                    tmem_ld4(tmem_ml + 4 * (chalf ^ 1), om, ol, pad0, pad1);
+                    float pm[4], pl[4], pad0, pad1;
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4) tmem_ld4(tmem_ml + 4 * k4, pm[k4], pl[k4], pad0, pad1);
                     tmem_wait_ld();
-                    const float mm = fmaxf(m, om);
-                    l = (m > -INFINITY ? l * fast_exp2(m - mm) : 0.f) + (om > -INFINITY ? ol * fast_exp2(om - mm) : 0.f);
-                    m = mm;
+                    m = fmaxf(fmaxf(pm[0], pm[1]), fmaxf(pm[2], pm[3]));      // part 0 always has key 0: finite
+                    l = 0.f;
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4) l += pm[k4] > -INFINITY ? pl[k4] * fast_exp2(pm[k4] - m) : 0.f;
                 }
-                const float lse = m + log2f(l);
-                // ---- pass B: normalised probabilities, P for the tensor core, pbar, activations ----
-                for (int kb = 0; kb < nkb && ok; ++kb, ++sb.count, ++tiles) {
+                // rows of padded head slots get lse = +inf: all their probabilities are exactly 0
+                const float lse = head_on ? m + log2f(l) : INFINITY;
+                // ---- pass B: normalised probabilities back into tensor memory, pbar, activations ----
+                for (int kb = 0; kb < nkb; ++kb, ++sb.count, ++tiles) {
                     const uint32_t buf = sb.stage(2);
-                    ok = named_barrier_and(2, kSoftmaxThreads,
-                                           wait_bar(&bars->s_full[buf], sb.parity(2), abort_flag, p.status, limit) &&
-                                               wait_bar(&bars->p_empty, (p_uses & 1u) ^ 1u, abort_flag, p.status, limit));
-                    if (!ok) break;
+                    wait_on(&bars->s_full[buf], sb.parity(2));
                     tmem_fence_after_sync();
                     uint32_t* act_t = act + (tiles & 1u) * kTile;
-#pragma unroll 1
-                    for (int c = 2 * chalf; c < 2 * chalf + 2; ++c) {
+                    {
                         float x[32];
-                        tmem_ld32(tmem_row + buf * 128 + c * 32, x);
+                        const uint32_t cols = tmem_row + kColS + buf * 128 + c * 32;
+                        tmem_ld32(cols, x);
                         tmem_wait_ld();
                         const int key0 = kb * kTile + c * 32;
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            x[i] = key0 + i <= pos ? fast_exp2(x[i] * p.scale_log2 - lse) : 0.f;
-                        // P as the K-major A operand of O += P V: row `row`, keys key0 .. key0 + 31 of this tile.
-                        // It enters the tensor core as two bf16 terms, p = hi + lo (16 mantissa bits): with one
-                        // term the weights would be off by up to 2^-9, more than the output tolerance allows
-                        // where large values cancel.
+                        for (int i = 0; i < 32; ++i) x[i] = fast_exp2(fmaf(x[i], p.scale_log2, -lse));
+                        if (key0 + 31 > pos) {      // the tile on the diagonal: keys beyond the row's position weigh nothing
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) x[i] = key0 + i <= pos ? x[i] : 0.f;
+                        }
+                        // P over the logits it came from, as the tensor-memory A operand of O += P V: two bf16
+                        // per column, the 32 keys of this chunk as 16 columns of hi terms then 16 of lo terms
+                        // (p = hi + lo, 16 mantissa bits: with one term the weights would be off by up to 2^-9,
+                        // more than the output tolerance allows where large values cancel).
                         {
-                            uint8_t* prow = p_s + (c >> 1) * kBoxBytes + row * 128;
+                            uint32_t hi[16], lo[16];
 #pragma unroll
-                            for (int ch = 0; ch < 4; ++ch) {
-                                uint32_t hi[4], lo[4];
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float a0 = x[8 * ch + 2 * e], a1 = x[8 * ch + 2 * e + 1];
-                                    hi[e] = pack_bf16(a0, a1);
-                                    lo[e] = pack_bf16(a0 - bf16_lo_as_float(hi[e]), a1 - bf16_hi_as_float(hi[e]));
-                                }
-                                const int chunk = (c & 1) * 4 + ch;
-                                uint8_t* dst = prow + ((chunk ^ (row & 7)) << 4);
-                                *reinterpret_cast<uint4*>(dst) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                                *reinterpret_cast<uint4*>(dst + kOperandBytes) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                            for (int e = 0; e < 16; ++e) {
+                                const float a0 = x[2 * e], a1 = x[2 * e + 1];
+                                hi[e] = pack_bf16(a0, a1);
+                                lo[e] = pack_bf16(a0 - bf16_lo_as_float(hi[e]), a1 - bf16_hi_as_float(hi[e]));
                             }
+                            tmem_st16(cols, hi);
+                            tmem_st16(cols + 16, lo);
                         }
                         // pbar: sum over the GP lanes of this position.  Every round halves what a lane keeps,
                         // so after log2(GP) rounds lane g holds 32 / GP columns summed over all heads.
-                        if (!head_on) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) x[i] = 0.f;
-                        }
                         int col0 = 0;               // first of the columns this lane ends up with
 #pragma unroll
                         for (int w = 1, half = 16; w < GP; w <<= 1, half >>= 1) {
@@ -487,20 +558,21 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             }
                         }
                     }
-                    fence_proxy_async();            // P is read by the tensor core through the async proxy
+                    tmem_wait_st();
                     tmem_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) {
-                        mbar_arrive(&bars->p_full);
+                        mbar_arrive(&bars->p_full[buf]);
                         mbar_arrive(&bars->s_empty[buf]);
                     }
-                    ++p_uses;
-                    // Eq. (1) for this tile's activations: thread `row` owns key column kb * 128 + row.
-                    named_barrier_sync(1, kSoftmaxThreads);
-                    const uint32_t bits = chalf == 0 ? act_t[row] : 0u;
+                    // Eq. (1) for this tile's activations.  The bits of the 32 columns of part c come from the four
+                    // warps of part c only, so those 128 threads synchronise among themselves (the parts stay
+                    // free to drift apart), and lane l of the part's first warp owns key column kb * 128 + 32 c + l.
+                    named_barrier_sync(3 + c, 128);
+                    const uint32_t bits = (warp & 3) == 0 ? act_t[c * 32 + lane] : 0u;
                     if (bits != 0u) {
-                        act_t[row] = 0u;
-                        const size_t s = srow + (size_t)kb * kTile + row;
+                        act_t[c * 32 + lane] = 0u;
+                        const size_t s = srow + (size_t)kb * kTile + c * 32 + lane;
                         int ts = p.ts[s], mri = p.mri[s];
                         uint32_t left = bits;
                         while (left != 0u) {        // positions of the tile in ascending order
@@ -514,32 +586,33 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         p.mri[s] = mri;
                     }
                 }
-                if (!ok) break;
-                // ---- the tile's attention output ----
-                ok = named_barrier_and(2, kSoftmaxThreads, wait_bar(&bars->o_full, o_uses & 1u, abort_flag, p.status, limit));
-                if (!ok) break;
+                // ---- the tile's attention output: bf16 into the tile's own Q slot (its MMAs are done), in the
+                // swizzled layout a TMA store expects; the producer warp sends it off before it refills the slot ----
+                wait_on(&bars->o_full, o_uses & 1u);
                 tmem_fence_after_sync();
-#pragma unroll 1
-                for (int c = 2 * chalf; c < 2 * chalf + 2; ++c) {
+                {
                     float x[32];
-                    tmem_ld32(tmem_row + 256 + c * 32, x);
+                    tmem_ld32(tmem_row + kColO + c * 32, x);
                     tmem_wait_ld();
-                    if (row_on) {
-                        __nv_bfloat16* orow = p.out + (((size_t)pos * p.units + u) * G + g) * kHeadDim + c * 32;
+                    tmem_fence_before_sync();
+                    uint8_t* orow = smem + kOffQ + qr.stage(2) * kOperandBytes + (c >> 1) * kBoxBytes + row * 128;
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
-                            uint4 w;
-                            w.x = pack_bf16(x[8 * ch + 0], x[8 * ch + 1]);
-                            w.y = pack_bf16(x[8 * ch + 2], x[8 * ch + 3]);
-                            w.z = pack_bf16(x[8 * ch + 4], x[8 * ch + 5]);
-                            w.w = pack_bf16(x[8 * ch + 6], x[8 * ch + 7]);
-                            *reinterpret_cast<uint4*>(orow + 8 * ch) = w;
-                        }
+                    for (int ch = 0; ch < 4; ++ch) {
+                        uint4 w;
+                        w.x = pack_bf16(x[8 * ch + 0], x[8 * ch + 1]);
+                        w.y = pack_bf16(x[8 * ch + 2], x[8 * ch + 3]);
+                        w.z = pack_bf16(x[8 * ch + 4], x[8 * ch + 5]);
+                        w.w = pack_bf16(x[8 * ch + 6], x[8 * ch + 7]);
+                        const int chunk = (c & 1) * 4 + ch;
+                        *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 7)) << 4)) = w;
                     }
                 }
-                tmem_fence_before_sync();
+                fence_proxy_async();                // the store reads shared memory through the async proxy
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&bars->o_empty);
+                if (lane == 0) {
+                    mbar_arrive(&bars->o_empty);
+                    mbar_arrive(&bars->out_ready[qr.stage(2)]);
+                }
                 ++o_uses;
             }
         }
@@ -549,7 +622,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     __syncthreads();
     if (warp == 0) {
         tmem_fence_after_sync();
-        tmem_dealloc(tmem_base, 512);
+        tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -581,11 +654,11 @@ bool make_map(CUtensorMap* map, const void* base, int rank, const cuuint64_t* di
 }
 
 template <int GP>
-cudaError_t launch_gp(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const PromptParams& p,
-                      int blocks, cudaStream_t stream) {
+cudaError_t launch_gp(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mo,
+                      const PromptParams& p, int blocks, cudaStream_t stream) {
     cudaError_t e = cudaFuncSetAttribute(prompt_kernel<GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPromptSmem);
     if (e != cudaSuccess) return e;
-    prompt_kernel<GP><<<blocks, kPromptThreads, kPromptSmem, stream>>>(mq, mk, mv, p);
+    prompt_kernel<GP><<<blocks, kPromptThreads, kPromptSmem, stream>>>(mq, mk, mv, mo, p);
     return cudaGetLastError();
 }
 
@@ -596,7 +669,7 @@ cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a
     int gp = 4;                 // head slots per position: at least 4, so that a tile's positions fit a 32-bit mask
     while (gp < G) gp *= 2;
     const int tq = kTile / gp;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, mo;
     {
         // q [P][units][G][128]: box = 64 dims x GP head slots x 1 unit x TQ positions -> rows (position, head slot);
         // head slots >= G and positions >= P are outside the tensor and read as zero.
@@ -604,6 +677,7 @@ cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a
         const cuuint64_t strides[3] = {(cuuint64_t)kRowBytes, (cuuint64_t)G * kRowBytes, (cuuint64_t)geo.units * G * kRowBytes};
         const cuuint32_t box[4] = {64, (cuuint32_t)gp, 1, (cuuint32_t)tq};
         if (!make_map(&mq, a.q, 4, dims, strides, box)) return cudaErrorInvalidValue;
+        if (!make_map(&mo, a.out, 4, dims, strides, box)) return cudaErrorInvalidValue;     // out is laid out like q
     }
     {
         // k, v [units][P][128]: box = 64 dims x 128 keys x 1 unit; keys >= P read as zero.
@@ -621,7 +695,6 @@ cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)kHeadDim);
     p.inv_group = 1.0f / (float)G;
     p.alpha = a.alpha;
-    p.out = reinterpret_cast<__nv_bfloat16*>(a.out);
     p.ts = st.ts;
     p.mri = st.mri;
     p.pbar = st.pbar;
@@ -631,7 +704,7 @@ cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a
     p.dump_count = a.dump_count;
     p.wait_limit_ns = a.wait_limit_ns;
     const int blocks = geo.units < num_sms ? geo.units : num_sms;
-    return gp == 4 ? launch_gp<4>(mq, mk, mv, p, blocks, stream) : launch_gp<8>(mq, mk, mv, p, blocks, stream);
+    return gp == 4 ? launch_gp<4>(mq, mk, mv, mo, p, blocks, stream) : launch_gp<8>(mq, mk, mv, mo, p, blocks, stream);
 }
 
 }  // namespace lzk
