@@ -164,19 +164,36 @@ __device__ void select_radix_unit(const int u, const Geometry& geo, const StateV
                 if (on && (int)(__ffs(peers) - 1) == lane) atomicAdd(&hist[digit], (unsigned)__popc(peers));
             }
             __syncthreads();
-            if (tid == 0) {
-                int cum = 0, digit = 0;
-                for (int b = 255; b >= 0; --b) {
-                    const int c = (int)hist[b];
-                    if (cum + c >= krem) {
-                        digit = b;
-                        break;
-                    }
-                    cum += c;
+            if (tid < 32) {
+                // The bin that holds the krem-th largest key, bins counted from the top: lane l sums bins
+                // 8 l .. 8 l + 7, a suffix scan over the lanes finds the lane, eight steps find the bin.
+                int c8[8], own = 0;
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    c8[b] = (int)hist[8 * lane + b];
+                    own += c8[b];
                 }
-                sh_prefix = prefix | ((unsigned long long)digit << shift);
-                sh_krem = krem - cum;
-                sh_done = hist[digit] == 1u;
+                int above = own;                   // inclusive suffix sum: this lane's bins and all higher ones
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_down_sync(0xffffffffu, above, o);
+                    if (lane + o < 32) above += v;
+                }
+                const bool here = above >= krem && above - own < krem;     // exactly one lane (krem >= 1 keys exist)
+                if (here) {
+                    int cum = above - own, digit = 8 * lane;
+#pragma unroll
+                    for (int b = 7; b >= 0; --b) {
+                        if (cum + c8[b] >= krem) {
+                            digit = 8 * lane + b;
+                            break;
+                        }
+                        cum += c8[b];
+                    }
+                    sh_prefix = prefix | ((unsigned long long)digit << shift);
+                    sh_krem = krem - cum;
+                    sh_done = hist[digit] == 1u;
+                }
             }
             __syncthreads();
             prefix = sh_prefix;

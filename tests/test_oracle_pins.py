@@ -436,3 +436,48 @@ def test_bf16_decoding():
     want = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).double().numpy()
     got = orc.bf16_bits_to_f64(bits)
     assert np.array_equal(got, want) and got[:3].tolist() == [1.0, -1.0, 2.0]
+
+
+def test_append_without_attention_keeps_the_same_cache():
+    """append() is attend() without the arithmetic: after any mix of the two, and across the storage's
+    growth steps and an eviction, both units hold the same tokens and give the same attention."""
+    rng = np.random.default_rng(31)
+    a = orc.OracleUnit(2, 8, budget=150, window=50, alpha=0.01, n_recent=10)
+    b = orc.OracleUnit(2, 8, budget=150, window=50, alpha=0.01, n_recent=10)
+    K0, V0 = rng.normal(size=(3, 8)), rng.normal(size=(3, 8))
+    a.prefill(K0, V0); b.prefill(K0, V0)
+    for t in range(1, 301):
+        q, k, v = rng.normal(size=(2, 8)), rng.normal(size=8), rng.normal(size=8)
+        out_a, pbar = a.attend(q, k, v)
+        if t % 7 == 0:
+            out_b, pbar_b = b.attend(q, k, v)
+            assert np.array_equal(out_a, out_b) and np.array_equal(pbar, pbar_b)
+        else:
+            b.append(k, v)
+        a.track(pbar); b.track(pbar)                 # the same probabilities drive both bookkeepings
+        assert (a.evict_if_due() is None) == (b.evict_if_due() is None)
+        assert a.n == b.n and a.t == b.t == t
+    assert a.n == 150 + 0 and np.array_equal(a.K, b.K) and np.array_equal(a.V, b.V)
+    assert np.array_equal(a.pos, b.pos) and np.array_equal(a.TS, b.TS) and np.array_equal(a.MRI, b.MRI)
+
+
+def test_observed_prompt_tracking_can_consume_supplied_probabilities():
+    """prefill_observed(pbar_rows=...): Eq. (1) over the prompt rows driven by given float32 rows.
+    Hand-worked: alpha = 0.3, rows (times -2, -1, 0) [0.9], [0.05, 0.95], [0.5, 0.1, 0.4]:
+    token 0 is active at -2 and again at 0 (MRI 2, TS 0); token 1 only at its own row; token 2 at its own."""
+    rng = np.random.default_rng(32)
+    Q, K, V = rng.normal(size=(3, 1, 4)), rng.normal(size=(3, 4)), rng.normal(size=(3, 4))
+    rows = np.zeros((3, 3), dtype=np.float32)
+    rows[0, :1], rows[1, :2], rows[2, :3] = [0.9], [0.05, 0.95], [0.5, 0.1, 0.4]
+    o = orc.OracleUnit(1, 4, budget=10, window=4, alpha=0.3)
+    outs = o.prefill_observed(Q, K, V, pbar_rows=rows)
+    assert o.TS.tolist() == [0, -1, 0] and o.MRI.tolist() == [2, 0, 0] and o.t == 0
+    # the attention itself is untouched by the override, and its own rows are kept for comparison
+    ref = orc.OracleUnit(1, 4, budget=10, window=4, alpha=0.3)
+    assert np.array_equal(outs, ref.prefill_observed(Q, K, V))
+    assert len(o.prompt_pbar) == 3 and np.allclose([r.sum() for r in o.prompt_pbar], 1.0)
+    # feeding a unit its own rows back changes nothing
+    own = np.zeros((3, 3)); [own.__setitem__((j, slice(0, j + 1)), ref.prompt_pbar[j]) for j in range(3)]
+    again = orc.OracleUnit(1, 4, budget=10, window=4, alpha=0.3)
+    again.prefill_observed(Q, K, V, pbar_rows=own)
+    assert np.array_equal(again.TS, ref.TS) and np.array_equal(again.MRI, ref.MRI)
