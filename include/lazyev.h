@@ -100,6 +100,12 @@ int lazyev_set_stages(lazyev_t* h, int stages);
  * a page of its own): 0 = choose automatically, else 1 or 2. */
 int lazyev_set_groups(lazyev_t* h, int groups);
 
+/* on != 0 (default): when a step's decode launch gives every thread block exactly one unit -- problems
+ * of up to one unit per SM, where a step is a few microseconds and launch latency decides -- the new
+ * token is written into the cache inside that launch (by the warp that streams the token's page)
+ * instead of by a launch of its own.  Results are identical either way. */
+int lazyev_set_fused_append(lazyev_t* h, int on);
+
 /* Bytes the caller must provide to lazyev_bind(); any output pointer may be NULL. */
 int lazyev_query_sizes(const lazyev_t* h, size_t* kv_bytes, size_t* state_bytes, size_t* scratch_bytes);
 

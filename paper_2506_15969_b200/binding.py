@@ -57,6 +57,7 @@ _PROTOS = {
     "lazyev_set_splits": [C.c_void_p, C.c_int],
     "lazyev_set_stages": [C.c_void_p, C.c_int],
     "lazyev_set_groups": [C.c_void_p, C.c_int],
+    "lazyev_set_fused_append": [C.c_void_p, C.c_int],
     "lazyev_query_sizes": [C.c_void_p, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)],
     "lazyev_bind": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "lazyev_set_page_table": [C.c_void_p, C.c_void_p],
@@ -190,6 +191,9 @@ class Engine:
 
     def set_groups(self, groups: int) -> None:
         self._check(lib().lazyev_set_groups(self._h, groups))
+
+    def set_fused_append(self, on: bool) -> None:
+        self._check(lib().lazyev_set_fused_append(self._h, int(on)))
 
     def set_page_table(self, table) -> None:
         arr = np.ascontiguousarray(np.asarray(table, dtype=np.int32))

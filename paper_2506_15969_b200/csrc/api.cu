@@ -29,6 +29,7 @@ struct lazyev {
     int prompt_dump_begin = 0, prompt_dump_count = 0;
     unsigned long long wait_limit_ns = 2000000000ull;   // bounded waits in the kernels give up after this long
     int stop_after_pages = -1;             // diagnostics: starve the decode kernel's page ring (-1: off)
+    int fuse_append = 1;                   // small problems: the append runs inside the decode launch
     // derived at bind
     bool bound = false, prefilled = false;
     int units = 0, group = 0, capacity = 0, pages_per_unit = 0;
@@ -299,9 +300,18 @@ struct HostPipe {
     uint8_t* out_host;
 };
 
+// The new token of a step (S1), when the step has one.
+struct NewToken {
+    const void* k;
+    const void* v;
+    int position;
+};
+
 // The decode launches of one step: attention of q over the first n cached tokens of every unit with
-// tracking at time t.
-int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPipe* pipe) {
+// tracking at time t.  `tok` (may be null) is the token to append at slot n - 1 first: as a launch of
+// its own, or -- when every block of the decode launch takes exactly one unit, the launch-latency-sized
+// problems -- inside the decode launch.
+int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPipe* pipe, const NewToken* tok = nullptr) {
     cudaError_t e = cudaSuccess;
     DecodeConfig c{h->units, h->group, h->pages_per_unit, h->capacity, h->alpha, h->force_splits, h->force_stages, h->force_groups,
                    h->wait_limit_ns, h->stop_after_pages};
@@ -382,6 +392,13 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
         return fail(h, LAZYEV_EINVAL, "no decode launch shape fits %d tokens per unit in shared memory", n);
     const int main_units = h->units - shape.tail_units;
     const int clusters = shape.clusters < main_units ? shape.clusters : main_units;
+    const bool fuse_append = tok && h->fuse_append && shape.tail_units == 0 && main_units <= clusters;
+    if (tok && !fuse_append) {
+        SpanGuard g(h, kSpanAppend, 0.0);
+        e = append_launch(geometry(h), h->pool, h->st, tok->k, tok->v, n - 1, t, tok->position, h->stream);
+        if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
+        h->launches += 1;
+    }
     {
         // algorithmic bytes: every cached K and V row read once, one probability written per token,
         // the queries read and the outputs written
@@ -435,7 +452,8 @@ int run_decode(lazyev_t* h, const void* q, void* out, int n, int t, const HostPi
             if (pipe) e = cudaStreamWaitEvent(h->stream, h->ev_in[r], 0);
             if (e != cudaSuccess) break;
             // a range of the main walk continues it; the last round's units are a walk of their own
-            DecodeArgs a{h->pool, h->st, q, out, n, t, begin[r], count[r], is_tail ? 0 : begin[r] / clusters};
+            DecodeArgs a{h->pool, h->st, q, out, n, t, begin[r], count[r], is_tail ? 0 : begin[r] / clusters,
+                         fuse_append ? tok->k : nullptr, fuse_append ? tok->v : nullptr, fuse_append ? tok->position : 0};
             const bool beside = is_tail && fork;
             if (e != cudaSuccess) break;
             e = decode_launch(c, is_tail ? tail_plan : plan, is_tail ? count[r] : (clusters < count[r] ? clusters : count[r]), a,
@@ -471,14 +489,8 @@ int run_step(lazyev_t* h, const void* q, const void* k_new, const void* v_new, v
         return fail(h, LAZYEV_EINVAL,
                     "step %d would evict over %d candidates, more than the selection supports; nothing was done", t,
                     n - h->n_recent - h->n_initial);
-    cudaError_t e;
-    {
-        SpanGuard g(h, kSpanAppend, 0.0);
-        e = append_launch(geometry(h), h->pool, h->st, k_new, v_new, n - 1, t, h->prefill + t - 1, h->stream);
-    }
-    if (e != cudaSuccess) return cuda_fail(h, e, "append kernel launch");
-    h->launches += 1;
-    const int rc = run_decode(h, q, out, n, t, pipe);
+    const NewToken tok{k_new, v_new, h->prefill + t - 1};
+    const int rc = run_decode(h, q, out, n, t, pipe, &tok);
     if (rc != LAZYEV_OK) return rc;
     h->t = t;
     h->n = n;
@@ -775,6 +787,12 @@ int lazyev_set_prompt_dump(lazyev_t* h, float* device_rows, int unit_begin, int 
     h->prompt_dump = device_rows;
     h->prompt_dump_begin = device_rows ? unit_begin : 0;
     h->prompt_dump_count = device_rows ? unit_count : 0;
+    return LAZYEV_OK;
+}
+
+int lazyev_set_fused_append(lazyev_t* h, int on) {
+    if (!h) return LAZYEV_EINVAL;
+    h->fuse_append = on != 0;
     return LAZYEV_OK;
 }
 

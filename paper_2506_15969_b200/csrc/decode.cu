@@ -49,7 +49,7 @@ struct Xchg {
 };
 
 struct DecodeParams {
-    const uint8_t* pool;
+    uint8_t* pool;
     const int32_t* page_table;
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
@@ -65,6 +65,12 @@ struct DecodeParams {
     unsigned long long wait_limit_ns;               // a wait that lasts this long is a failure, not a delay
     int stop_after_pages;                           // diagnostics: the producer issues no copy beyond this many (-1: off)
     int rounds_before;                              // rounds of the round-robin walk that earlier launches of this step took
+    // Step S1 inside this launch (small problems: one launch less per step): the new token's K / V rows
+    // [units][128] bf16, written into slot n - 1 by the block that streams the slot's page.
+    const uint4* k_new;                             // nullptr: the append ran as a launch of its own
+    const uint4* v_new;
+    int32_t* pos;
+    int append_position;
 };
 
 constexpr float kRaiseMargin = 8.f;                // log2 units a logit may exceed the softmax reference by
@@ -171,11 +177,31 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                     }
                     int32_t pp = __shfl_sync(0xffffffffu, entry, j);
                     if (pc >= (uint32_t)NS) wait_phase(&empty[stage], parity, abort_flag, p.status, p.wait_limit_ns);
-                    if (lane == 0) {
-                        if (pp < 0 || pp >= p.total_pages) {
-                            atomicOr(p.status, kStatusBadIndex);
-                            pp = 0;
+                    if (pp < 0 || pp >= p.total_pages) {
+                        if (lane == 0) atomicOr(p.status, kStatusBadIndex);
+                        pp = 0;
+                    }
+                    if (p.k_new != nullptr && pg0 + base + j == (p.n - 1) / kPageTokens &&
+                        in_bounds(p.n >= 1 && p.n <= p.capacity, p.status)) {
+                        // The new token (Section 4: TS = t, MRI = 0) goes into slot n - 1 of this page before the
+                        // page is streamed: lanes 0..15 move the K row's chunks, lanes 16..31 the V row's.  The
+                        // bulk copy below reads global memory through the async proxy, so the rows are fenced
+                        // across the proxies first; the state words become visible to the consumer warps with
+                        // the page (the barrier's release / acquire).
+                        const int r = (p.n - 1) % kPageTokens, c = lane & 15;
+                        const uint4 v = (lane < 16 ? p.k_new : p.v_new)[(size_t)u * kChunksPerRow + c];
+                        uint8_t* row = p.pool + (size_t)pp * kPageBytes + (lane < 16 ? 0 : kPageHalfBytes) + r * kRowBytes;
+                        *reinterpret_cast<uint4*>(row + swz_chunk(c, r) * 16) = v;
+                        if (lane == 0) {
+                            const size_t sl = (size_t)u * p.capacity + (p.n - 1);
+                            p.ts[sl] = p.t;
+                            p.mri[sl] = 0;
+                            p.pos[sl] = p.append_position;
                         }
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                        __syncwarp();
+                    }
+                    if (lane == 0) {
                         mbar_arrive_expect_tx(&full[stage], kPageBytes);
                         bulk_load(ring + (size_t)stage * kPageBytes, p.pool + (size_t)pp * kPageBytes, kPageBytes,
                                   &full[stage]);
@@ -725,7 +751,11 @@ cudaError_t decode_max_clusters(const DecodePlan& plan, int* clusters) {
 cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clusters, const DecodeArgs& a,
                           cudaStream_t stream) {
     DecodeParams p;
-    p.pool = a.pool;
+    p.pool = const_cast<uint8_t*>(a.pool);
+    p.k_new = reinterpret_cast<const uint4*>(a.k_new);
+    p.v_new = reinterpret_cast<const uint4*>(a.v_new);
+    p.pos = a.state.pos;
+    p.append_position = a.append_position;
     p.page_table = a.state.page_table;
     p.q = reinterpret_cast<const __nv_bfloat16*>(a.q);
     p.out = reinterpret_cast<__nv_bfloat16*>(a.out);

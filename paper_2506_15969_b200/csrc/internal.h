@@ -30,6 +30,9 @@ struct DecodeArgs {
     int t;                 // this decode step
     int unit_begin, unit_count;   // the units this launch covers
     int rounds_before;            // whole rounds of the same walk done by earlier launches (0 for a walk of its own)
+    const void* k_new;            // non-null: the launch also appends the new token (slot n - 1, TS = t, MRI = 0)
+    const void* v_new;
+    int append_position;
 };
 
 // Deepest ring and the shared-memory layout for n cached tokens and a cluster of `splits` blocks;

@@ -515,6 +515,37 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_recovers():
     assert du["device_status"] == 0 and used.info().evictions == fresh.info().evictions + 0
 
 
+@pytest.mark.parametrize("splits", [0, 1, 3])
+def test_append_inside_the_decode_launch_matches_the_separate_launch(splits):
+    """Small problems write the new token inside the decode launch (one launch less per step); with the
+    switch off the append is a launch of its own.  Same outputs, state and cache, bit for bit, across a
+    page boundary and two evictions; and one launch per step less."""
+    from tests.harness import make_engine
+    cfg = traces.tiny_config(prefill=100)
+    gen = traces.TraceGen(cfg, 27, device="cuda")
+    fused, plain = make_engine(cfg), make_engine(cfg)
+    plain.set_fused_append(False)
+    for e in (fused, plain):
+        e.set_splits(splits)
+    k, v = gen.prefill()
+    shape = (cfg.layers, cfg.batch, cfg.kv_heads, cfg.prefill, 128)
+    fused.prefill(k.view(shape), v.view(shape)); plain.prefill(k.view(shape), v.view(shape))
+    out_f = torch.empty(cfg.layers, cfg.batch, cfg.q_heads, 128, dtype=torch.bfloat16, device="cuda")
+    out_p = torch.empty_like(out_f)
+    l0 = (fused.info().launches, plain.info().launches)
+    for _ in range(4):
+        q, kn, vn = gen.steps(32)
+        for s in range(32):
+            fused.decode_step(q[s], kn[s], vn[s], out_f)
+            plain.decode_step(q[s], kn[s], vn[s], out_p)
+            assert torch.equal(out_f, out_p)
+    df, dp = fused.dump_state(kv=True), plain.dump_state(kv=True)
+    for key in ("pos", "ts", "mri", "pbar", "k", "v"):
+        assert np.array_equal(df[key], dp[key]), key
+    assert df["device_status"] == 0 and fused.info().evictions == plain.info().evictions == 3
+    assert (plain.info().launches - l0[1]) - (fused.info().launches - l0[0]) == 128
+
+
 def test_library_flavour_is_the_one_the_environment_asks_for():
     assert bool(binding.lib().lazyev_build_flags() & 1) == binding.debug_bounds_requested()
 
@@ -529,7 +560,7 @@ def test_range_checked_build_runs_the_lockstep_tests_clean():
         pytest.skip("already inside the range-checked run")
     env = dict(os.environ, LAZYEV_DEBUG_BOUNDS="1")
     here = os.path.dirname(os.path.abspath(__file__))
-    sel = ("lockstep_with_evictions or random_shapes or many_units or group_sizes or observed_prompt or "
+    sel = ("lockstep_with_evictions or random_shapes or many_units or group_sizes or observed_prompt or append_inside or "
            "partly_filled or protected_tokens or dynamic_budget or window_of_one or library_flavour or "
            "long_contexts or histogram")
     res = subprocess.run([sys.executable, "-m", "pytest", os.path.join(here, "test_gpu_parity.py"),
