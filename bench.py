@@ -40,8 +40,8 @@ FALLBACK_HBM_GBS = 6650.0
 # units x tokens, so a full launch is scaled by its algorithmic bytes.  Valid only for the kernel
 # sources it was taken on.
 NCU_DECODE_CAPTURE = {
-    "traffic_per_algorithmic_byte": 1.0076,
-    "sha256": {"decode.cu": "d739e597f7047acf3fdc725e9f668ebab9c5300f20f42208c6054b7e068ba0c8",
+    "traffic_per_algorithmic_byte": 1.0075,
+    "sha256": {"decode.cu": "beb36a72346a7192ab168577ec8e0b6725be576bd8085f6f1285ca6f6c50f6ba",
                "common.cuh": "bd1929d12b75ef1f2ea3bd900d3f93f7a39494c3ab52ff7dd9fe31945b995fd2"},
 }
 

@@ -412,7 +412,8 @@ typedef struct lazyev_profile {
 int lazyev_set_profiling(lazyev_t* h, int on);
 int lazyev_get_profile(lazyev_t* h, lazyev_profile_t* out, int reset);
 
-/* Waits for the stream and reads the device status word: 0, EDEVICE or ECUDA. */
+/* Waits for the stream (and for steps queued with lazyev_decode_step_host_async) and reads the device
+ * status word: 0, EDEVICE or ECUDA. */
 int lazyev_synchronize(lazyev_t* h);
 
 /* Frees the host-side handle.  Device memory stays with the caller. */

@@ -710,9 +710,17 @@ int lazyev_prefill(lazyev_t* h, const void* k, const void* v, int n_tokens) {
     return LAZYEV_OK;
 }
 
+namespace {
+int host_wait(lazyev_t* h, int allowed);
+}
+
 int lazyev_reset(lazyev_t* h) {
     if (!h) return LAZYEV_EINVAL;
     if (!h->bound) return fail(h, LAZYEV_ESTATE, "reset before bind");
+    if (h->copy_in) {                       // steps queued through the asynchronous host entry point finish first
+        const int rc = host_wait(h, 0);
+        if (rc != LAZYEV_OK) return rc;
+    }
     // Old rows stay in the pool: slots past n are masked, they only have to be finite.  The state arrays
     // are rewritten by the next prompt load and by every append; the device status word is cleared.
     cudaError_t e = cudaMemsetAsync(h->st.status, 0, 64, h->stream);
@@ -1207,11 +1215,16 @@ int lazyev_get_profile(lazyev_t* h, lazyev_profile_t* out, int reset) {
 int lazyev_synchronize(lazyev_t* h) {
     if (!h) return LAZYEV_EINVAL;
     if (!h->bound) return fail(h, LAZYEV_ESTATE, "synchronize before bind");
+    if (h->copy_in) {
+        const int rc = host_wait(h, 0);
+        if (rc != LAZYEV_OK) return rc;
+    }
     return check_device_status(h);
 }
 
 int lazyev_destroy(lazyev_t* h) {
     if (!h) return LAZYEV_EINVAL;
+    if (h->copy_in) host_wait(h, 0);        // no copy of ours may still be writing the caller's host buffers
     for (const lazyev::Span& sp : h->pending) {
         cudaEventDestroy(sp.start);
         cudaEventDestroy(sp.stop);
