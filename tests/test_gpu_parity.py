@@ -278,7 +278,8 @@ def test_mri_histogram_and_quantile_match_the_oracle():
 
 
 @pytest.mark.parametrize("mode", [binding.PROMPT_TILED, binding.PROMPT_REPLAY])
-@pytest.mark.parametrize("prefill,q_heads,kv_heads", [(150, 8, 2), (333, 8, 2), (512, 10, 2), (700, 7, 1), (2048, 6, 2)])
+@pytest.mark.parametrize("prefill,q_heads,kv_heads", [(150, 8, 2), (333, 8, 2), (512, 10, 2), (700, 7, 1), (2048, 6, 2),
+                                                     (97, 2, 2), (260, 16, 2)])
 def test_observed_prompt_then_decode(prefill, q_heads, kv_heads, mode):
     """lazyev_prefill_observed: causal prompt attention with tracking from the first token, by the tiled
     tensor-core kernel and by the row-by-row replay through the decode kernel, each against the oracle
@@ -299,34 +300,41 @@ def test_observed_prompt_then_decode(prefill, q_heads, kv_heads, mode):
     assert rep.evictions == 2
 
 
-def test_tiled_prompt_kernel_agrees_with_the_replay():
+@pytest.mark.parametrize("batch,layers,prefill", [(3, 2, 400), (40, 4, 300)])
+def test_tiled_prompt_kernel_agrees_with_the_replay(batch, layers, prefill):
     """The two implementations of the prompt pass on the same prompt: attention outputs equal to within
-    bf16 rounding of the inputs to P V, probabilities to float32 rounding; the statistics they produce
-    may differ only for tokens whose probability came within that rounding of the threshold."""
+    bf16 rounding, probabilities to float32 rounding; the statistics they produce may differ only for
+    tokens whose probability came within that rounding of the threshold.  The second case has 320 units:
+    every block of the tiled kernel walks two or three units, so its rings, Q slots and output stores run
+    across unit boundaries."""
     from tests.harness import make_engine
-    cfg = traces.tiny_config(prefill=400, budget=500, window=32, alpha=0.02, batch=3, layers=2)
+    cfg = traces.tiny_config(prefill=prefill, budget=prefill + 100, window=32, alpha=0.02, batch=batch, layers=layers)
     gen = traces.TraceGen(cfg, 23, device="cuda")
     k, v = gen.prefill()
     shape = (cfg.layers, cfg.batch, cfg.kv_heads, cfg.prefill, 128)
     g = torch.Generator().manual_seed(5)
     q = torch.randn(cfg.prefill, cfg.units, cfg.group, 128, generator=g).to(torch.bfloat16).cuda()
+    dumped = min(cfg.units, 24)                               # per-row probabilities of the last units only
     res = {}
     for mode in (binding.PROMPT_TILED, binding.PROMPT_REPLAY):
         eng = make_engine(cfg)
         eng.set_prompt_mode(mode)
-        rows = torch.zeros(cfg.units, cfg.prefill, cfg.prefill, dtype=torch.float32, device="cuda")
-        out = torch.empty(cfg.prefill, cfg.units, cfg.group, 128, dtype=torch.bfloat16, device="cuda")
-        eng.set_prompt_dump(rows, 0, cfg.units)
+        rows = torch.zeros(dumped, cfg.prefill, cfg.prefill, dtype=torch.float32, device="cuda")
+        out = torch.zeros(cfg.prefill, cfg.units, cfg.group, 128, dtype=torch.bfloat16, device="cuda")
+        eng.set_prompt_dump(rows, cfg.units - dumped, dumped)
         eng.prefill_observed(q, k.view(shape), v.view(shape), out)
         eng.synchronize()
         res[mode] = (out.float().cpu(), rows.cpu(), eng.dump_state())
-        assert eng.info().launches == (3 if mode == binding.PROMPT_TILED else 2 + cfg.prefill)
+        if cfg.units <= 148:
+            assert eng.info().launches == (3 if mode == binding.PROMPT_TILED else 2 + cfg.prefill)
     (o_t, r_t, d_t), (o_r, r_r, d_r) = res[binding.PROMPT_TILED], res[binding.PROMPT_REPLAY]
-    assert (o_t - o_r).abs().max() <= 2e-3 + 1e-2 * o_r.abs().max()
+    assert ((o_t - o_r).abs() <= 4e-3 + 2e-2 * o_r.abs()).all()            # two implementations, each within the oracle's bar
     assert (r_t - r_r).abs().max() <= 2e-6
-    near = ((r_r - cfg.threshold).abs() <= 2e-6).any(dim=1).numpy()            # [units, tokens]: ever close to alpha
+    assert np.abs(d_t["pbar"] - d_r["pbar"]).max() <= 2e-6
+    near = ((r_r - cfg.threshold).abs() <= 2e-6).any(dim=1).numpy()            # [dumped units, tokens]: ever close to alpha
     same = (d_t["ts"] == d_r["ts"]) & (d_t["mri"] == d_r["mri"])
-    assert (same | near).all() and same.mean() > 0.99
+    assert (same[cfg.units - dumped:] | near).all() and same.mean() > 0.99
+    assert d_t["device_status"] == 0 and d_r["device_status"] == 0
 
 
 def test_reset_then_a_new_sequence_gives_the_same_results_as_a_fresh_handle():
