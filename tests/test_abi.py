@@ -94,3 +94,32 @@ def test_capacity_grows_with_a_long_prompt():
     lib.lazyev_get_info(h, C.byref(info))
     assert info.capacity == 1152 and info.pages_per_unit == 18
     lib.lazyev_destroy(h)
+
+
+def test_diagnostic_and_mode_setters_validate_arguments():
+    """Host-side checks of the switches that need no device: wait limit, prompt mode, per-row dump range,
+    page-ring starvation, in-launch append; and the calls that need a bound handle say so."""
+    lib = binding.lib()
+    rc, h = create(2, 8, 2, 128, 512, 128, 1e-3)
+    assert rc == binding.OK
+    assert lib.lazyev_set_wait_limit(h, 0.004) == binding.OK
+    assert lib.lazyev_set_wait_limit(h, 0.0) == binding.EINVAL and lib.lazyev_set_wait_limit(h, 1e9) == binding.EINVAL
+    assert lib.lazyev_set_wait_limit(h, float("nan")) == binding.EINVAL
+    assert lib.lazyev_set_prompt_mode(h, binding.PROMPT_REPLAY) == binding.OK
+    assert lib.lazyev_set_prompt_mode(h, 7) == binding.EINVAL
+    assert lib.lazyev_debug_starve_page_ring(h, 3) == binding.OK and lib.lazyev_debug_starve_page_ring(h, -1) == binding.OK
+    assert lib.lazyev_debug_starve_page_ring(h, -2) == binding.EINVAL
+    assert lib.lazyev_set_fused_append(h, 0) == binding.OK and lib.lazyev_set_fused_append(h, 1) == binding.OK
+    fake = C.c_void_p(256)                                     # never dereferenced: only the range is checked here
+    assert lib.lazyev_set_prompt_dump(h, fake, 0, 4) == binding.OK           # units = 2 layers x 1 batch x 2 heads
+    assert lib.lazyev_set_prompt_dump(h, fake, 3, 2) == binding.EINVAL
+    assert lib.lazyev_set_prompt_dump(h, None, 0, 0) == binding.OK
+    assert lib.lazyev_host_wait(h, 2) == binding.EINVAL and lib.lazyev_host_wait(h, 0) == binding.OK
+    counters = binding.Counters()
+    assert lib.lazyev_get_counters(h, C.byref(counters)) == binding.ESTATE   # before bind
+    assert lib.lazyev_synchronize(h) == binding.ESTATE and lib.lazyev_reset(h) == binding.ESTATE
+    assert lib.lazyev_copy_state(h, h) == binding.EINVAL
+    rc2, h2 = create(2, 8, 2, 128, 512, 128, 1e-3)
+    assert lib.lazyev_copy_state(h2, h) == binding.ESTATE      # neither handle is bound
+    assert lib.lazyev_build_flags() in (0, 1)
+    assert lib.lazyev_destroy(h) == binding.OK and lib.lazyev_destroy(h2) == binding.OK
