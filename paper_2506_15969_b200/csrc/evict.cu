@@ -77,7 +77,8 @@ __device__ __forceinline__ int block_sum(int v, int* warp_sums) {
 struct SelectShared {
     unsigned int hist[256];
     unsigned long long prefix;
-    int krem, first, done;
+    unsigned long long surv[kSelThreads];          // the keys still in the race once they are few
+    int krem, first, done, n_surv;
     int warp_sums[kSelThreads / 32];
 };
 
@@ -108,27 +109,27 @@ __device__ void select_radix_unit(const int u, const Geometry& geo, const StateV
     const unsigned lt = (1u << lane) - 1u;
 
     // Scores are >= 0, so their IEEE bit patterns order like unsigned integers; a score of exactly 0
-    // (never re-activated) has key 0.  Whether a score is exactly 0 follows from the integers alone:
-    // with MRI = 0 it is 0 unless the elapsed time is 0; with MRI != 0 the H1 term 2 / (1 + exp(d / MRI))
-    // is positive as long as the exponential is finite (d / MRI <= 700 is far inside that range; beyond
-    // it the score is evaluated to see); H2 alone (mode 2) is 0 exactly for MRI <= 1.  So the first pass
-    // needs no floating point: it stores 0 or the packed pair (d, MRI) with the top bit set, and counts.
+    // (never re-activated) has key 0.  Units come here because more of their scores are non-zero than
+    // tokens are kept, so Eq. (2) is evaluated in fp64 for every candidate (tokens with MRI = 0 take the
+    // short way through it); eight steps' loads are in flight before the first evaluation.
     int nonzero = 0;
-    for (int i0 = seg_b; i0 < seg_e; i0 += 32) {
-        const int i = i0 + lane;
-        if (i < seg_e) {
-            const int m = mri[i], d = a.t - ts[i];
-            bool zero;
-            if (a.score_mode == 2)
-                zero = m <= 1;
-            else if (m == 0)
-                zero = d != 0;
-            else if ((long long)d > 700ll * m)
-                zero = score_with_table(d, m, a.score_mode, a.h2_table, a.h2_entries) == 0.0;
-            else
-                zero = false;
-            keys[i] = zero ? 0ull : (1ull << 63) | ((unsigned long long)(unsigned)d << 32) | (unsigned)m;
-            nonzero += !zero;
+    for (int i0 = seg_b; i0 < seg_e; i0 += 8 * 32) {
+        int mm[8], tt[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = i0 + 32 * q + lane;
+            mm[q] = i < seg_e ? __ldg(mri + i) : 0;
+            tt[q] = i < seg_e ? __ldg(ts + i) : 0;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int i = i0 + 32 * q + lane;
+            if (i < seg_e) {
+                const unsigned long long key = (unsigned long long)__double_as_longlong(
+                    score_with_table(a.t - tt[q], mm[q], a.score_mode, a.h2_table, a.h2_entries));
+                keys[i] = key;
+                nonzero += key != 0ull;
+            }
         }
     }
     if (tid == 0) sh_first = ncand;
@@ -138,18 +139,10 @@ __device__ void select_radix_unit(const int u, const Geometry& geo, const StateV
     unsigned long long kth = 0;
     int krem = k - nonzero;
     if (nonzero > k) {
-        // More non-zero scores than tokens to keep: the k-th score has to be found.  Eq. (2) in fp64 for
-        // every non-zero candidate (most of them in this regime, so the warps stay converged) ...
-        for (int i = tid; i < ncand; i += kSelThreads) {
-            const unsigned long long packed = keys[i];
-            if (packed != 0ull)
-                keys[i] = (unsigned long long)__double_as_longlong(score_with_table(
-                    (int)((packed >> 32) & 0x7FFFFFFFull), (int)(packed & 0xFFFFFFFFull), a.score_mode, a.h2_table, a.h2_entries));
-        }
-        __syncthreads();
-        // ... then a radix select over the non-zero keys, most significant byte first.  The histogram is built with
+        // More non-zero scores than tokens to keep: the k-th score is found by a radix select over the
+        // non-zero keys, most significant byte first.  The histogram is built with
         // one shared-memory atomic per distinct digit and warp (scores cluster in a few exponents), and
-        // the passes stop as soon as the k-th key is alone in its bin.
+        // the passes stop as soon as the k-th key's bin holds at most one key per thread.
         unsigned long long prefix = 0, mask = 0;
         krem = k;
         for (int shift = 56; shift >= 0; shift -= 8) {
@@ -192,7 +185,7 @@ __device__ void select_radix_unit(const int u, const Geometry& geo, const StateV
                     }
                     sh_prefix = prefix | ((unsigned long long)digit << shift);
                     sh_krem = krem - cum;
-                    sh_done = hist[digit] == 1u;
+                    sh_done = hist[digit] <= (unsigned)kSelThreads;
                 }
             }
             __syncthreads();
@@ -202,12 +195,34 @@ __device__ void select_radix_unit(const int u, const Geometry& geo, const StateV
             if (sh_done) break;                    // uniform: read from shared memory after the barrier
         }
         kth = prefix;
-        if (mask != ~0ull) {                       // stopped early: the only key with this prefix is the k-th
+        if (mask != ~0ull) {
+            // Stopped early: at most one key per thread shares the prefix.  They are gathered, and every
+            // thread ranks its own among them: the k-th is the key with fewer than krem keys above it and
+            // at least krem keys at or above it.
+            if (tid == 0) sh.n_surv = 0;
             __syncthreads();
-            for (int i = tid; i < ncand; i += kSelThreads)
-                if (keys[i] != 0ull && (keys[i] & mask) == prefix) sh_prefix = keys[i];
+            for (int i = tid; i < ncand; i += kSelThreads) {
+                const unsigned long long key = keys[i];
+                if (key != 0ull && (key & mask) == prefix) sh.surv[atomicAdd(&sh.n_surv, 1)] = key;
+            }
+            __syncthreads();
+            const int n_surv = sh.n_surv;
+            if (tid < n_surv) {
+                const unsigned long long mine = sh.surv[tid];
+                int above = 0, equal = 0;
+                for (int j = 0; j < n_surv; ++j) {
+                    const unsigned long long other = sh.surv[j];
+                    above += other > mine;
+                    equal += other == mine;
+                }
+                if (above < krem && krem <= above + equal) {       // equal keys all write the same two values
+                    sh_prefix = mine;
+                    sh_krem = krem - above;
+                }
+            }
             __syncthreads();
             kth = sh_prefix;
+            krem = sh_krem;
         }
     }
     // keep every key > kth, and `krem` of the keys == kth
