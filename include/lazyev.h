@@ -29,7 +29,7 @@
  *             bits), which makes a linear bulk copy of a page land in shared
  *             memory free of ldmatrix bank conflicts.  Slot i of unit u lives
  *             in physical page page_table[u][i / 64], row i % 64.
- *   state   : page table, and per unit and slot: TS (int32), MRI (int32),
+ *   state   : page table, and per unit and slot: the pair (TS, MRI) as two int32 side by side,
  *             original position (int32), last probability (float32).
  *   scratch : eviction source lists, staging for the host-buffer entry point, score
  *             staging for lazyev_dump_state, the MRI histogram.

@@ -115,7 +115,7 @@ void derive(lazyev_t* h) {
 
 struct Sizes {
     size_t kv, state, scratch;
-    size_t off_ts, off_mri, off_pos, off_pbar, off_status;                          // inside state
+    size_t off_tsm, off_pos, off_pbar, off_status;                                  // inside state
     size_t off_first, off_rlist, off_q, off_k, off_v, off_out, off_score, off_hist, off_h2;    // inside scratch
 };
 
@@ -124,10 +124,8 @@ Sizes sizes_of(const lazyev_t* h) {
     const size_t slots = (size_t)h->units * h->capacity;
     s.kv = (size_t)h->units * h->pages_per_unit * kPageBytes;
     size_t off = align_up((size_t)h->units * h->pages_per_unit * sizeof(int32_t), 256);
-    s.off_ts = off;
-    off += align_up(slots * 4, 256);
-    s.off_mri = off;
-    off += align_up(slots * 4, 256);
+    s.off_tsm = off;                       // (TS, MRI) pairs
+    off += align_up(slots * 8, 256);
     s.off_pos = off;
     off += align_up(slots * 4, 256);
     s.off_pbar = off;
@@ -643,8 +641,7 @@ int lazyev_bind(lazyev_t* h, void* kv_pool, void* state, void* scratch, void* cu
     h->pool = (uint8_t*)kv_pool;
     uint8_t* sp = (uint8_t*)state;
     h->st.page_table = (int32_t*)sp;
-    h->st.ts = (int32_t*)(sp + s.off_ts);
-    h->st.mri = (int32_t*)(sp + s.off_mri);
+    h->st.tsm = (int2*)(sp + s.off_tsm);
     h->st.pos = (int32_t*)(sp + s.off_pos);
     h->st.pbar = (float*)(sp + s.off_pbar);
     h->st.status = (int32_t*)(sp + s.off_status);
@@ -1064,10 +1061,18 @@ int lazyev_dump_state(lazyev_t* h, lazyev_dump_t* d) {
     int32_t status = 0;
     e = cudaMemcpyAsync(&status, h->st.status, sizeof(status), cudaMemcpyDeviceToHost, h->stream);
     if (e == cudaSuccess && d->pos) e = cudaMemcpyAsync(d->pos, h->st.pos + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
-    if (e == cudaSuccess && d->ts) e = cudaMemcpyAsync(d->ts, h->st.ts + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
-    if (e == cudaSuccess && d->mri) e = cudaMemcpyAsync(d->mri, h->st.mri + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
+    std::vector<int2> pairs;               // TS and MRI sit interleaved on the device
+    if (e == cudaSuccess && (d->ts || d->mri)) {
+        pairs.resize(count);
+        e = cudaMemcpyAsync(pairs.data(), h->st.tsm + first, count * sizeof(int2), cudaMemcpyDeviceToHost, h->stream);
+    }
     if (e == cudaSuccess && d->pbar) e = cudaMemcpyAsync(d->pbar, h->st.pbar + first, count * 4, cudaMemcpyDeviceToHost, h->stream);
+    if (e == cudaSuccess && !pairs.empty()) e = cudaStreamSynchronize(h->stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "state download");
+    for (size_t i = 0; i < pairs.size(); ++i) {
+        if (d->ts) d->ts[i] = pairs[i].x;
+        if (d->mri) d->mri[i] = pairs[i].y;
+    }
     if (d->score) {
         const Geometry geo = geometry(h);
         for (int u0 = 0; u0 < d->unit_count; u0 += kScoreStageUnits) {
@@ -1122,8 +1127,13 @@ int lazyev_load_state(lazyev_t* h, const lazyev_dump_t* d, int prefill) {
         return fail(h, LAZYEV_EINVAL, "snapshot sizes out of range (n = %d, capacity here = %d)", d->n, h->capacity);
     const size_t scap = (size_t)d->capacity, width = (size_t)d->n * 4;
     cudaError_t e = cudaMemcpy2DAsync(h->st.pos, (size_t)h->capacity * 4, d->pos, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
-    if (e == cudaSuccess) e = cudaMemcpy2DAsync(h->st.ts, (size_t)h->capacity * 4, d->ts, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
-    if (e == cudaSuccess) e = cudaMemcpy2DAsync(h->st.mri, (size_t)h->capacity * 4, d->mri, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
+    std::vector<int2> pairs((size_t)h->units * d->n);      // interleaved (TS, MRI), rows of n
+    for (int u = 0; u < h->units; ++u)
+        for (int i = 0; i < d->n; ++i)
+            pairs[(size_t)u * d->n + i] = make_int2(d->ts[(size_t)u * scap + i], d->mri[(size_t)u * scap + i]);
+    if (e == cudaSuccess)
+        e = cudaMemcpy2DAsync(h->st.tsm, (size_t)h->capacity * 8, pairs.data(), (size_t)d->n * 8, (size_t)d->n * 8, h->units,
+                              cudaMemcpyHostToDevice, h->stream);
     if (e == cudaSuccess && d->pbar) e = cudaMemcpy2DAsync(h->st.pbar, (size_t)h->capacity * 4, d->pbar, scap * 4, width, h->units, cudaMemcpyHostToDevice, h->stream);
     if (e != cudaSuccess) return cuda_fail(h, e, "state upload");
     // K / V rows: swizzled into pages on the host, one page per copy

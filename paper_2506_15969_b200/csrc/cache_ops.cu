@@ -14,8 +14,7 @@ __global__ void init_state_kernel(Geometry geo, StateView st) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total_slots; i += stride) {
         if (i < total_pages) st.page_table[i] = (int32_t)i;      // identity: unit u owns pages [u*ppu, (u+1)*ppu)
         if (i < 16) st.status[i] = 0;
-        st.ts[i] = 0;
-        st.mri[i] = 0;
+        st.tsm[i] = make_int2(0, 0);
         st.pos[i] = 0;
         st.pbar[i] = 0.f;
     }
@@ -40,8 +39,7 @@ __global__ void prefill_kernel(Geometry geo, uint8_t* pool, StateView st, const 
             const size_t s = (size_t)u * geo.capacity + i;
             // Prompt tokens start at MRI = 0 (Section 4) and TS = 0, or, when the prompt is going to be
             // replayed with tracking, at their own time ts_first + i (the last prompt row is time 0).
-            st.ts[s] = ts_first == INT_MIN ? 0 : ts_first + i;
-            st.mri[s] = 0;
+            st.tsm[s] = make_int2(ts_first == INT_MIN ? 0 : ts_first + i, 0);
             st.pos[s] = i;
         }
     }
@@ -62,8 +60,7 @@ __global__ void append_kernel(Geometry geo, uint8_t* pool, StateView st, const u
     *reinterpret_cast<uint4*>(row + swz_chunk(c, r) * 16) = *src;
     if (lane == 0) {
         const size_t s = (size_t)u * geo.capacity + slot;
-        st.ts[s] = t;              // a token is born active at its own step
-        st.mri[s] = 0;
+        st.tsm[s] = make_int2(t, 0);      // a token is born active at its own step, with MRI = 0
         st.pos[s] = position;
     }
 }

@@ -41,8 +41,8 @@ __host__ __device__ __forceinline__ int swz_chunk(int c, int r) { return c ^ (r 
 // Per-slot state arrays of one handle.
 struct StateView {
     int32_t* page_table;   // [units][pages_per_unit]
-    int32_t* ts;           // [units][capacity]
-    int32_t* mri;          // [units][capacity]
+    int2* tsm;             // [units][capacity]: x = TS (last activation), y = MRI -- one 8-byte word per
+                           // token, so that Eq. (1) is one load and one store and the selection reads one stream
     int32_t* pos;          // [units][capacity]
     float* pbar;           // [units][capacity]
     int32_t* status;       // [16]

@@ -54,8 +54,7 @@ struct DecodeParams {
     const __nv_bfloat16* q;
     __nv_bfloat16* out;
     float* pbar;
-    int32_t* ts;
-    int32_t* mri;
+    int2* tsm;                                      // (TS, MRI) per token
     int32_t* status;
     int unit_begin, unit_end, group, pages_per_unit, capacity, total_pages;     // this launch walks units [begin, end)
     int n, t;
@@ -194,8 +193,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                         *reinterpret_cast<uint4*>(row + swz_chunk(c, r) * 16) = v;
                         if (lane == 0) {
                             const size_t sl = (size_t)u * p.capacity + (p.n - 1);
-                            p.ts[sl] = p.t;
-                            p.mri[sl] = 0;
+                            p.tsm[sl] = make_int2(p.t, 0);
                             p.pos[sl] = p.append_position;
                         }
                         asm volatile("fence.proxy.async.global;" ::: "memory");
@@ -320,16 +318,15 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
         // found and its result is used one emit_previous call later (a page's worth of work), so the
         // update never stalls the warp that holds a ring stage; at most one token per half is pending.
         long long pend_idx0 = -1, pend_idx1 = -1;
-        int32_t pend_ts0 = 0, pend_ts1 = 0;
+        int2 pend_old0 = make_int2(0, 0), pend_old1 = make_int2(0, 0);
         auto retire_pending = [&]() {
             if (pend_idx0 >= 0) {
-                atomicMax(&p.mri[pend_idx0], p.t - pend_ts0);      // MRI = max(MRI, t - TS)
-                p.ts[pend_idx0] = p.t;                             // TS = t
+                // MRI = max(MRI, t - TS), TS = t: the token belongs to this lane alone, one 8-byte store
+                p.tsm[pend_idx0] = make_int2(p.t, max(pend_old0.y, p.t - pend_old0.x));
                 pend_idx0 = -1;
             }
             if (pend_idx1 >= 0) {
-                atomicMax(&p.mri[pend_idx1], p.t - pend_ts1);
-                p.ts[pend_idx1] = p.t;
+                p.tsm[pend_idx1] = make_int2(p.t, max(pend_old1.y, p.t - pend_old1.x));
                 pend_idx1 = -1;
             }
         };
@@ -354,7 +351,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                     p.pbar[row + i0] = pb;
                     if (pb >= p.alpha) {
                         pend_idx0 = (long long)(row + i0);
-                        pend_ts0 = p.ts[row + i0];
+                        pend_old0 = p.tsm[row + i0];
                     }
                 }
                 if (tok0 + i1 < p.n) {
@@ -362,7 +359,7 @@ __global__ void __launch_bounds__((4 * NG + 1) * 32, 1) decode_kernel(const Deco
                     p.pbar[row + i1] = pb;
                     if (pb >= p.alpha) {
                         pend_idx1 = (long long)(row + i1);
-                        pend_ts1 = p.ts[row + i1];
+                        pend_old1 = p.tsm[row + i1];
                     }
                 }
             }
@@ -760,8 +757,7 @@ cudaError_t decode_launch(const DecodeConfig& c, const DecodePlan& plan, int clu
     p.q = reinterpret_cast<const __nv_bfloat16*>(a.q);
     p.out = reinterpret_cast<__nv_bfloat16*>(a.out);
     p.pbar = a.state.pbar;
-    p.ts = a.state.ts;
-    p.mri = a.state.mri;
+    p.tsm = a.state.tsm;
     p.status = a.state.status;
     p.unit_begin = a.unit_begin;
     p.unit_end = a.unit_begin + a.unit_count;

@@ -94,8 +94,7 @@ __device__ void select_radix_unit(const int u, const Geometry& geo, const StateV
     const int S = a.n_initial, R = a.n_recent;
     const int ncand = a.n - R - S;                 // unprotected slots [S, n - R)
     const int k = a.budget - R - S;                // how many of them stay
-    const int32_t* ts = st.ts + (size_t)u * geo.capacity + S;
-    const int32_t* mri = st.mri + (size_t)u * geo.capacity + S;
+    const int2* tsm = st.tsm + (size_t)u * geo.capacity + S;       // (TS, MRI) of the candidates
     int32_t* src = a.src + (size_t)u * a.budget;
     if (!in_bounds(S >= 0 && R >= 0 && ncand > 0 && k >= 0 && k <= ncand && a.n <= geo.capacity && a.budget <= a.n, st.status))
         return;
@@ -118,8 +117,9 @@ __device__ void select_radix_unit(const int u, const Geometry& geo, const StateV
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             const int i = i0 + 32 * q + lane;
-            mm[q] = i < seg_e ? __ldg(mri + i) : 0;
-            tt[q] = i < seg_e ? __ldg(ts + i) : 0;
+            const int2 w = i < seg_e ? __ldg(tsm + i) : make_int2(0, 0);
+            tt[q] = w.x;
+            mm[q] = w.y;
         }
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -322,8 +322,7 @@ __global__ void __launch_bounds__(kSelThreads) select_fast_kernel(Geometry geo, 
     const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int S = a.n_initial, R = a.n_recent;
     const int ncand = a.n - R - S, k = a.budget - R - S;
-    const int32_t* ts = st.ts + (size_t)u * geo.capacity + S;
-    const int32_t* mri = st.mri + (size_t)u * geo.capacity + S;
+    const int2* tsm = st.tsm + (size_t)u * geo.capacity + S;       // (TS, MRI) of the candidates
     int32_t* src = a.src + (size_t)u * a.budget;
     if (!in_bounds(S >= 0 && R >= 0 && ncand > 0 && k >= 0 && k <= ncand && a.n <= geo.capacity && a.budget <= a.n, st.status))
         return;
@@ -332,7 +331,7 @@ __global__ void __launch_bounds__(kSelThreads) select_fast_kernel(Geometry geo, 
     const int nsteps = (seg_e - seg_b + 31) / 32;
     const unsigned lt = (1u << lane) - 1u;
 
-    // (eight steps at a time: all sixteen loads of a lane are in flight before the first ballot, which
+    // (eight steps at a time: all eight loads of a lane are in flight before the first ballot, which
     // is what keeps this pass bound by bandwidth and not by one memory latency per step)
     int nz_warp = 0;
     for (int s0 = 0; s0 < nsteps; s0 += 8) {
@@ -341,8 +340,9 @@ __global__ void __launch_bounds__(kSelThreads) select_fast_kernel(Geometry geo, 
         for (int q = 0; q < 8; ++q) {
             const int i = seg_b + (s0 + q) * 32 + lane;
             const bool in = s0 + q < nsteps && i < seg_e;
-            mm[q] = in ? __ldg(mri + i) : 0;
-            tt[q] = in ? __ldg(ts + i) : a.t - 1;      // outside: MRI = 0, elapsed 1 -> a zero score
+            const int2 w = in ? __ldg(tsm + i) : make_int2(a.t - 1, 0);    // outside: MRI = 0, elapsed 1 -> a zero score
+            tt[q] = w.x;
+            mm[q] = w.y;
         }
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -504,10 +504,10 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(Geometry ge
                     page_ptr(pool, page_of(srow[i] / kPageTokens)) + half + (srow[i] % kPageTokens) * kRowBytes;
                 val[i] = *reinterpret_cast<const uint4*>(row + cp * 16);
             }
-        int s_ts = 0, s_mri = 0, s_pos = 0;
+        int2 s_tsm = make_int2(0, 0);
+        int s_pos = 0;
         if (s_from >= 0) {
-            s_ts = st.ts[sbase + s_from];
-            s_mri = st.mri[sbase + s_from];
+            s_tsm = st.tsm[sbase + s_from];
             s_pos = st.pos[sbase + s_from];
         }
         // next tile's source indices: in flight together with this tile's rows
@@ -528,8 +528,7 @@ __global__ void __launch_bounds__(kCompactThreads, 3) compact_kernel(Geometry ge
             srow[i] = srow_next[i];
         }
         if (s_from >= 0) {
-            st.ts[sbase + d0 + tid] = s_ts;
-            st.mri[sbase + d0 + tid] = s_mri;
+            st.tsm[sbase + d0 + tid] = s_tsm;
             st.pos[sbase + d0 + tid] = s_pos;
         }
         s_from = s_from_next;
@@ -542,7 +541,8 @@ __global__ void score_kernel(Geometry geo, StateView st, int unit_begin, int uni
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const int u = (int)(i / geo.capacity), s = (int)(i % geo.capacity);
         const size_t g = (size_t)(unit_begin + u) * geo.capacity + s;
-        out[i] = s < n ? score_fn(t - st.ts[g], st.mri[g], mode) : 0.0;
+        const int2 w = st.tsm[g];
+        out[i] = s < n ? score_fn(t - w.x, w.y, mode) : 0.0;
     }
 }
 
@@ -561,11 +561,11 @@ __global__ void __launch_bounds__(256) mri_histogram_kernel(Geometry geo, StateV
     __syncthreads();
     const int lane = threadIdx.x & 31;
     for (int u = unit_begin + blockIdx.x; u < unit_begin + unit_count; u += gridDim.x) {
-        const int32_t* mri = st.mri + (size_t)u * geo.capacity;
+        const int2* tsm = st.tsm + (size_t)u * geo.capacity;
         for (int i0 = 0; i0 < n; i0 += blockDim.x) {
             const int i = i0 + threadIdx.x;
             const bool on = i < n;
-            const int v = on ? mri[i] : -1;
+            const int v = on ? tsm[i].y : -1;
             const int b = v < 0 ? 0 : min(v, bins - 1);
             // most tokens share one value (0): one atomic per distinct value and warp
             const unsigned peers = __match_any_sync(0xffffffffu, on ? b : -1);

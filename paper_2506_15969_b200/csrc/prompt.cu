@@ -70,8 +70,7 @@ struct Bars {                                       // mbarriers
 struct PromptParams {
     int units, group, P, capacity;
     float scale_log2, inv_group, alpha;
-    int32_t* ts;
-    int32_t* mri;
+    int2* tsm;                                      // (TS, MRI) per token
     float* pbar;
     int32_t* status;
     float* dump;                                    // optional: [dump_count][P][P] probabilities per prompt row
@@ -573,7 +572,8 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     if (bits != 0u) {
                         act_t[c * 32 + lane] = 0u;
                         const size_t s = srow + (size_t)kb * kTile + c * 32 + lane;
-                        int ts = p.ts[s], mri = p.mri[s];
+                        const int2 old = p.tsm[s];
+                        int ts = old.x, mri = old.y;
                         uint32_t left = bits;
                         while (left != 0u) {        // positions of the tile in ascending order
                             const int b = __ffs(left) - 1;
@@ -582,8 +582,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             mri = max(mri, time - ts);          // MRI = max(MRI, t - TS)
                             ts = time;                          // TS = t
                         }
-                        p.ts[s] = ts;
-                        p.mri[s] = mri;
+                        p.tsm[s] = make_int2(ts, mri);
                     }
                 }
                 // ---- the tile's attention output: bf16 into the tile's own Q slot (its MMAs are done), in the
@@ -695,8 +694,7 @@ cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)kHeadDim);
     p.inv_group = 1.0f / (float)G;
     p.alpha = a.alpha;
-    p.ts = st.ts;
-    p.mri = st.mri;
+    p.tsm = st.tsm;
     p.pbar = st.pbar;
     p.status = st.status;
     p.dump = a.dump;
