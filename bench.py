@@ -40,9 +40,9 @@ FALLBACK_HBM_GBS = 6650.0
 # units x tokens, so a full launch is scaled by its algorithmic bytes.  Valid only for the kernel
 # sources it was taken on.
 NCU_DECODE_CAPTURE = {
-    "traffic_per_algorithmic_byte": 1.0075,
-    "sha256": {"decode.cu": "beb36a72346a7192ab168577ec8e0b6725be576bd8085f6f1285ca6f6c50f6ba",
-               "common.cuh": "bd1929d12b75ef1f2ea3bd900d3f93f7a39494c3ab52ff7dd9fe31945b995fd2"},
+    "traffic_per_algorithmic_byte": 1.0072,
+    "sha256": {"decode.cu": "d503c2c87321f96c31e2e309b6839b3a37a429614323ee1bb163f2251c1c05a9",
+               "common.cuh": "38bde61410b93126cf44ed1a98971cc365c31108efb5043fc9500d293d16e3f1"},
 }
 
 
