@@ -279,7 +279,7 @@ def test_mri_histogram_and_quantile_match_the_oracle():
 
 @pytest.mark.parametrize("mode", [binding.PROMPT_TILED, binding.PROMPT_REPLAY])
 @pytest.mark.parametrize("prefill,q_heads,kv_heads", [(150, 8, 2), (333, 8, 2), (512, 10, 2), (700, 7, 1), (2048, 6, 2),
-                                                     (97, 2, 2), (260, 16, 2)])
+                                                     (97, 2, 2), (260, 16, 2), (17, 8, 2)])
 def test_observed_prompt_then_decode(prefill, q_heads, kv_heads, mode):
     """lazyev_prefill_observed: causal prompt attention with tracking from the first token, by the tiled
     tensor-core kernel and by the row-by-row replay through the decode kernel, each against the oracle
@@ -294,7 +294,7 @@ def test_observed_prompt_then_decode(prefill, q_heads, kv_heads, mode):
     ls = lockstep(cfg, seed=17, sample_units=sample, observed=True, prompt_mode=mode)
     d = ls.eng.dump_state(0, 1)
     assert (d["ts"][0] >= np.arange(prefill) - (prefill - 1)).all() and d["ts"][0].max() == 0
-    assert (d["mri"][0] > 0).sum() >= 5                       # prompt tokens were re-activated
+    assert (d["mri"][0] > 0).sum() >= min(5, prefill // 8)    # prompt tokens were re-activated
     rep = ls.run(100, check_every=1 if prefill < 1000 else 8)
     ls.assert_ok()
     assert rep.evictions == 2
