@@ -481,3 +481,54 @@ def test_observed_prompt_tracking_can_consume_supplied_probabilities():
     again = orc.OracleUnit(1, 4, budget=10, window=4, alpha=0.3)
     again.prefill_observed(Q, K, V, pbar_rows=own)
     assert np.array_equal(again.TS, ref.TS) and np.array_equal(again.MRI, ref.MRI)
+
+
+# ---- property-based pins (hypothesis): the bookkeeping against a per-token restatement of Eq. (1) ----
+from hypothesis import given, settings, strategies as st_
+
+
+@settings(max_examples=60, deadline=None)
+@given(st_.integers(1, 6), st_.integers(1, 40), st_.integers(0, 2 ** 32 - 1))
+def test_track_equals_a_per_token_state_machine(n_tokens, steps, seed):
+    """Eq. (1) token by token: a token's MRI is the largest gap between consecutive activations
+    (its birth counts as one), its TS the last of them.  Random activation patterns through track()
+    against that restatement computed from the whole history at once."""
+    rng = np.random.default_rng(seed)
+    alpha = 0.5
+    u = orc.OracleUnit(1, 4, budget=1000, window=500, alpha=alpha)
+    u.prefill(np.zeros((n_tokens, 4)), np.zeros((n_tokens, 4)))
+    history = []                                     # per step: activation mask over the tokens alive then
+    for t in range(1, steps + 1):
+        u.append(np.zeros(4), np.zeros(4))
+        act = rng.random(u.n) < 0.3
+        pbar = np.where(act, 0.9, 0.1).astype(np.float32)
+        got = u.track(pbar)
+        assert np.array_equal(got, act)
+        history.append(act)
+    for i in range(u.n):
+        birth = 0 if i < n_tokens else i - n_tokens + 1          # prompt tokens start at TS = 0
+        times = [birth] + [t for t in range(max(birth, 1), steps + 1) if history[t - 1][i]]
+        gaps = [b - a for a, b in zip(times, times[1:])]
+        assert u.TS[i] == times[-1] and u.MRI[i] == max(gaps + [0])
+
+
+@settings(max_examples=40, deadline=None)
+@given(st_.integers(0, 2 ** 32 - 1))
+def test_eviction_invariants_on_random_runs(seed):
+    """Whatever the probabilities: the cache holds exactly B_t tokens after an eviction and never more than
+    B + W, positions stay strictly increasing, the R newest and S oldest tokens always survive, and what is
+    kept scores at least as high as what goes (Eq. (evic) generalised)."""
+    rng = np.random.default_rng(seed)
+    W = int(rng.integers(1, 9)); R = int(rng.integers(1, W + 1)); S = int(rng.integers(0, 3))
+    B = int(rng.integers(max(W, R + S) + 1, 40)); P = int(rng.integers(1, 30))
+    u = orc.OracleUnit(2, 4, budget=B, window=W, alpha=float(rng.choice([0.0, 0.02, 0.2, 2.0])), n_recent=R, n_initial=S)
+    u.prefill(rng.normal(size=(P, 4)), rng.normal(size=(P, 4)))
+    for t in range(1, 5 * W + 7):
+        n_before = u.n
+        _, _, info = u.step(rng.normal(size=(2, 4)) * 3, rng.normal(size=4), rng.normal(size=4))
+        assert (t % W == 0 and n_before + 1 > B) == (info is not None)
+        if info is not None:
+            assert u.n == B and info["kept_min"] >= info["evicted_max"]
+            assert u.pos[-R:].tolist() == list(range(P + t - R, P + t))
+            assert u.pos[:S].tolist() == list(range(S))         # the oldest S tokens are never evicted
+        assert u.n <= max(B, P) + W and np.all(np.diff(u.pos) > 0) and u.t == t
