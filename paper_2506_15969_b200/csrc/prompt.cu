@@ -197,6 +197,36 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
     return true;
 }
 
+// Two fp32 lanes per instruction (packed .f32x2 arithmetic) and the three-input maximum: the softmax warps
+// are bound by the number of instructions they issue per logit, not by any one pipe.  Each lane rounds
+// exactly like the scalar instruction, so results do not depend on which form is used.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t r, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 // One use of a barrier pair in a ring: which stage and which parity a counter of uses maps to.
 struct Ring {
     uint32_t count = 0;
@@ -433,6 +463,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
             const bool dumping = p.dump != nullptr && u >= p.dump_begin && u < p.dump_begin + p.dump_count;
             for (int qt = 0; qt < n_qt; ++qt, ++qr.count) {
                 const int pos = qt * TQ + jj;
+                const int warp_last_pos = qt * TQ + (32 * (warp & 3)) / GP + 32 / GP - 1;      // of this warp's 32 rows
                 const int nkb = key_tiles(qt);
                 // ---- pass A: exact log-sum-exp of the row (log2 domain) ----
                 float m = -INFINITY, l = 0.f;
@@ -440,7 +471,9 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     const uint32_t buf = sb.stage(2);
                     wait_on(&bars->s_full[buf], sb.parity(2));
                     tmem_fence_after_sync();
-                    {
+                    // On the diagonal tile a whole chunk of 32 keys can lie beyond every position of this warp's rows:
+                    // nothing of it counts (with short prompts that is a third of all the chunks).
+                    if (kb * kTile + c * 32 <= warp_last_pos) {
                         float x[32];
                         tmem_ld32(tmem_row + kColS + buf * 128 + c * 32, x);
                         tmem_wait_ld();
@@ -449,28 +482,31 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
 #pragma unroll
                             for (int i = 0; i < 32; ++i) x[i] = key0 + i <= pos ? x[i] : -INFINITY;
                         }
-                        float c0 = fmaxf(x[0], x[1]), c1 = fmaxf(x[2], x[3]), c2 = fmaxf(x[4], x[5]), c3 = fmaxf(x[6], x[7]);
+                        float c0 = fmax3(x[0], x[1], x[2]), c1 = fmax3(x[3], x[4], x[5]);
 #pragma unroll
-                        for (int i = 8; i < 32; i += 4) {
-                            c0 = fmaxf(c0, x[i]);
-                            c1 = fmaxf(c1, x[i + 1]);
-                            c2 = fmaxf(c2, x[i + 2]);
-                            c3 = fmaxf(c3, x[i + 3]);
+                        for (int i = 6; i < 30; i += 4) {
+                            c0 = fmax3(c0, x[i], x[i + 1]);
+                            c1 = fmax3(c1, x[i + 2], x[i + 3]);
                         }
-                        const float cmax = fmaxf(fmaxf(c0, c1), fmaxf(c2, c3)) * p.scale_log2;     // the scale is positive
+                        const float cmax = fmax3(c0, c1, fmaxf(x[30], x[31])) * p.scale_log2;      // the scale is positive
                         if (cmax > m) {
                             l *= fast_exp2(m - cmax);     // m = -inf only while l = 0
                             m = cmax;
                         }
                         if (m > -INFINITY) {
-                            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+                            const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), minus_m = pack2(-m, -m);
+                            uint64_t l01 = pack2(0.f, 0.f), l23 = l01;
 #pragma unroll
                             for (int i = 0; i < 32; i += 4) {
-                                l0 += fast_exp2(fmaf(x[i], p.scale_log2, -m));
-                                l1 += fast_exp2(fmaf(x[i + 1], p.scale_log2, -m));
-                                l2 += fast_exp2(fmaf(x[i + 2], p.scale_log2, -m));
-                                l3 += fast_exp2(fmaf(x[i + 3], p.scale_log2, -m));
+                                float e0, e1, e2, e3;
+                                unpack2(fma2(pack2(x[i], x[i + 1]), scale2, minus_m), e0, e1);
+                                unpack2(fma2(pack2(x[i + 2], x[i + 3]), scale2, minus_m), e2, e3);
+                                l01 = add2(l01, pack2(fast_exp2(e0), fast_exp2(e1)));
+                                l23 = add2(l23, pack2(fast_exp2(e2), fast_exp2(e3)));
                             }
+                            float l0, l1, l2, l3;
+                            unpack2(l01, l0, l1);
+                            unpack2(l23, l2, l3);
                             l += (l0 + l1) + (l2 + l3);
                         }
                     }
@@ -502,14 +538,32 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     wait_on(&bars->s_full[buf], sb.parity(2));
                     tmem_fence_after_sync();
                     uint32_t* act_t = act + (tiles & 1u) * kTile;
-                    {
+                    // the state words of the key column this lane owns, requested before the tile's arithmetic so
+                    // that they are there when the activations are applied (only this thread ever writes them)
+                    const int own_key = kb * kTile + c * 32 + lane;
+                    int2 own = make_int2(0, 0);
+                    if ((warp & 3) == 0 && own_key < P) own = p.tsm[srow + own_key];
+                    const uint32_t cols = tmem_row + kColS + buf * 128 + c * 32;
+                    if (kb * kTile + c * 32 > warp_last_pos) {
+                        // a chunk beyond all of this warp's positions: P = 0, nothing to add up or to test
+                        const uint32_t zero[16] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+                        tmem_st16(cols, zero);
+                        tmem_st16(cols + 16, zero);
+                    } else {
                         float x[32];
-                        const uint32_t cols = tmem_row + kColS + buf * 128 + c * 32;
                         tmem_ld32(cols, x);
                         tmem_wait_ld();
                         const int key0 = kb * kTile + c * 32;
+                        {
+                            const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), minus_lse = pack2(-lse, -lse);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) x[i] = fast_exp2(fmaf(x[i], p.scale_log2, -lse));
+                            for (int i = 0; i < 32; i += 2) {
+                                float e0, e1;
+                                unpack2(fma2(pack2(x[i], x[i + 1]), scale2, minus_lse), e0, e1);
+                                x[i] = fast_exp2(e0);
+                                x[i + 1] = fast_exp2(e1);
+                            }
+                        }
                         if (key0 + 31 > pos) {      // the tile on the diagonal: keys beyond the row's position weigh nothing
 #pragma unroll
                             for (int i = 0; i < 32; ++i) x[i] = key0 + i <= pos ? x[i] : 0.f;
@@ -524,7 +578,9 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             for (int e = 0; e < 16; ++e) {
                                 const float a0 = x[2 * e], a1 = x[2 * e + 1];
                                 hi[e] = pack_bf16(a0, a1);
-                                lo[e] = pack_bf16(a0 - bf16_lo_as_float(hi[e]), a1 - bf16_hi_as_float(hi[e]));
+                                float r0, r1;
+                                unpack2(sub2(pack2(a0, a1), pack2(bf16_lo_as_float(hi[e]), bf16_hi_as_float(hi[e]))), r0, r1);
+                                lo[e] = pack_bf16(r0, r1);
                             }
                             tmem_st16(cols, hi);
                             tmem_st16(cols + 16, lo);
@@ -536,10 +592,12 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         for (int w = 1, half = 16; w < GP; w <<= 1, half >>= 1) {
                             const bool upper = (lane & w) != 0;
 #pragma unroll
-                            for (int i = 0; i < half; ++i) {
-                                const float send = upper ? x[i] : x[i + half];
-                                const float keep = upper ? x[i + half] : x[i];
-                                x[i] = keep + __shfl_xor_sync(0xffffffffu, send, w);
+                            for (int i = 0; i < half; i += 2) {
+                                const float send0 = upper ? x[i] : x[i + half], send1 = upper ? x[i + 1] : x[i + 1 + half];
+                                const float keep0 = upper ? x[i + half] : x[i], keep1 = upper ? x[i + 1 + half] : x[i + 1];
+                                unpack2(add2(pack2(keep0, keep1), pack2(__shfl_xor_sync(0xffffffffu, send0, w),
+                                                                        __shfl_xor_sync(0xffffffffu, send1, w))),
+                                        x[i], x[i + 1]);
                             }
                             col0 += upper ? half : 0;
                         }
@@ -571,9 +629,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     const uint32_t bits = (warp & 3) == 0 ? act_t[c * 32 + lane] : 0u;
                     if (bits != 0u) {
                         act_t[c * 32 + lane] = 0u;
-                        const size_t s = srow + (size_t)kb * kTile + c * 32 + lane;
-                        const int2 old = p.tsm[s];
-                        int ts = old.x, mri = old.y;
+                        int ts = own.x, mri = own.y;
                         uint32_t left = bits;
                         while (left != 0u) {        // positions of the tile in ascending order
                             const int b = __ffs(left) - 1;
@@ -582,7 +638,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             mri = max(mri, time - ts);          // MRI = max(MRI, t - TS)
                             ts = time;                          // TS = t
                         }
-                        p.tsm[s] = make_int2(ts, mri);
+                        p.tsm[srow + own_key] = make_int2(ts, mri);
                     }
                 }
                 // ---- the tile's attention output: bf16 into the tile's own Q slot (its MMAs are done), in the
