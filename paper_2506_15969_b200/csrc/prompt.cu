@@ -549,6 +549,13 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         const uint32_t zero[16] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
                         tmem_st16(cols, zero);
                         tmem_st16(cols + 16, zero);
+                        tmem_wait_st();
+                        tmem_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) {
+                            mbar_arrive(&bars->p_full[buf]);
+                            mbar_arrive(&bars->s_empty[buf]);
+                        }
                     } else {
                         float x[32];
                         tmem_ld32(cols, x);
@@ -585,6 +592,15 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             tmem_st16(cols, hi);
                             tmem_st16(cols + 16, lo);
                         }
+                        // P is in place and the logits are in registers: hand the buffer to the tensor core now,
+                        // the head sums below need nothing from tensor memory
+                        tmem_wait_st();
+                        tmem_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) {
+                            mbar_arrive(&bars->p_full[buf]);
+                            mbar_arrive(&bars->s_empty[buf]);
+                        }
                         // pbar: sum over the GP lanes of this position.  Every round halves what a lane keeps,
                         // so after log2(GP) rounds lane g holds 32 / GP columns summed over all heads.
                         int col0 = 0;               // first of the columns this lane ends up with
@@ -614,13 +630,6 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                                 }
                             }
                         }
-                    }
-                    tmem_wait_st();
-                    tmem_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive(&bars->p_full[buf]);
-                        mbar_arrive(&bars->s_empty[buf]);
                     }
                     // Eq. (1) for this tile's activations.  The bits of the 32 columns of part c come from the four
                     // warps of part c only, so those 128 threads synchronise among themselves (the parts stay
