@@ -189,6 +189,8 @@ int lazyev_set_wait_limit(lazyev_t* h, double seconds);
  * limit and flag the device status word.  Nothing faults: the kernel ends by itself, and the
  * outputs and statistics of that step are undefined (lazyev_reset() before the handle is used
  * again).  Honoured by launches with one block per unit (lazyev_set_splits(h, 1)); -1 = off.
+ * The tiled prompt kernel of lazyev_prefill_observed() honours it too: the thread that feeds a
+ * block's ring of key tiles issues no copy beyond its first `pages` key tiles, with the same outcome.
  */
 int lazyev_debug_starve_page_ring(lazyev_t* h, int pages);
 

@@ -753,6 +753,7 @@ int lazyev_prefill_observed(lazyev_t* h, const void* q, const void* k, const voi
         a.dump_begin = h->prompt_dump_begin;
         a.dump_count = h->prompt_dump_count;
         a.wait_limit_ns = h->wait_limit_ns;
+        a.stop_after_tiles = h->stop_after_pages;
         e = prompt_launch(geometry(h), h->st, a, h->num_sms, h->stream);
         if (e != cudaSuccess) return cuda_fail(h, e, "prompt kernel launch");
         h->launches += 1;

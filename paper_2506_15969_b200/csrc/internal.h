@@ -62,6 +62,7 @@ struct PromptArgs {
     float* dump;           // optional [dump_count][P][P] probabilities per prompt row
     int dump_begin, dump_count;
     unsigned long long wait_limit_ns;
+    int stop_after_tiles;  // diagnostics: starve the K-tile ring (-1: off)
 };
 // TS / MRI of the prompt tokens must already hold their starting values (TS = own time, MRI = 0).
 cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a, int num_sms, cudaStream_t stream);

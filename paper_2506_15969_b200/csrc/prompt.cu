@@ -76,6 +76,7 @@ struct PromptParams {
     float* dump;                                    // optional: [dump_count][P][P] probabilities per prompt row
     int dump_begin, dump_count;
     unsigned long long wait_limit_ns;
+    int stop_after_tiles;                           // diagnostics: the producer stops after this many K tiles (-1: off)
 };
 
 // ---- PTX wrappers used only here ------------------------------------------------------------------
@@ -171,6 +172,29 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t leading_by
 // Instruction descriptor: fp32 accumulator, bf16 A and B, M = 128, N = 128; b_mn_major = B is MN-major.
 __host__ __device__ constexpr uint32_t instr_desc(bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// Has the phase with this parity completed?  Never suspends the thread (try_wait may, for a while).
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Sleep until the phase completes or about `ns` nanoseconds have passed, whichever is first: a wait that
+// leaves the issue slots to the other warps of the scheduler, unlike a polling loop.
+__device__ __forceinline__ void mbar_nap(uint64_t* bar, uint32_t parity, uint32_t ns) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%0], %1, %2;\n\t}" ::"r"(smem_u32(bar)),
+        "r"(parity), "r"(ns)
+        : "memory");
 }
 
 // Bounded wait on an mbarrier phase; on time-out the abort flag and the device status word are set
@@ -322,6 +346,10 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                     for (int pass = 0; pass < 2 && ok; ++pass) {
                         for (int kb = 0; kb < nkb; ++kb) {
                             const uint32_t ks = kr.stage(kKStages);
+                            // diagnostics: no copy beyond the first stop_after_tiles K tiles -- the other roles wait
+                            // for a tile that never comes, give up after the wait limit and flag the status word
+                            ok = p.stop_after_tiles < 0 || (int)kr.count < p.stop_after_tiles;
+                            if (!ok) break;
                             ok = wait_bar(&bars->k_empty[ks], kr.parity(kKStages) ^ 1u, abort_flag, p.status, limit);
                             if (!ok) break;
                             uint8_t* k_s = smem + kOffK + ks * kOperandBytes;
@@ -368,51 +396,44 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
     } else if (warp == kSoftmaxWarps + 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            Ring kr, vr, qr, sb;                    // K, V, Q uses and S buffer uses
-            uint32_t p_cnt[2] = {0, 0}, o_uses = 0;
-            bool ok = true;
+            // Two cursors walk the same sequence of (unit, query tile) pairs.  The S cursor issues the logits
+            // products -- per query tile one per key tile for pass A, then one per key tile for pass B; job j goes
+            // to S buffer j % 2 -- and the O cursor issues O += P V behind the softmax warps.  The S cursor may be
+            // up to one job past the O cursor's job: the job after that would overwrite the P the O cursor is
+            // about to read.  Its run-ahead crosses query tile and unit boundaries, so the first logits of the next
+            // query tile are computed while the softmax warps still work on the last key tile of this one.  The
+            // thread polls both cursors and issues whichever has everything it needs; it never blocks on one
+            // while the other could go (a late Q or K tile must not hold back the product that completes O).
+            Ring kr, vr, sq, sb;                    // K and V ring uses, query tiles begun by the S cursor, S jobs issued
+            uint32_t p_cnt0 = 0, p_cnt1 = 0, o_uses = 0;
             const uint32_t idesc_s = instr_desc(false), idesc_o = instr_desc(true);
             const uint32_t tmem_o = tmem_base + kColO;
+            int s_u = blockIdx.x, s_qt = 0, s_pass = 0, s_kb = 0, s_nkb = key_tiles(0);
+            bool s_more = s_u < p.units;
+            int o_u = blockIdx.x, o_qt = 0, o_kb = 0, o_nkb = key_tiles(0);
+            bool o_more = o_u < p.units;
+            uint32_t o_job = (uint32_t)o_nkb;       // the pass B job whose P the O cursor's next product reads
             uint32_t q_addr = 0;
-            // S[buffer] = Q K^T for the next K tile of the ring; the K stage is free once these MMAs are done
-            auto issue_s = [&]() -> bool {
-                const uint32_t ks = kr.stage(kKStages), buf = sb.stage(2);
-                if (!(wait_bar(&bars->k_full[ks], kr.parity(kKStages), abort_flag, p.status, limit) &&
-                      wait_bar(&bars->s_empty[buf], sb.parity(2) ^ 1u, abort_flag, p.status, limit)))
-                    return false;
-                tmem_fence_after_sync();
-                const uint32_t k_addr = smem_u32(smem + kOffK + ks * kOperandBytes);
-#pragma unroll
-                for (int s8 = 0; s8 < 8; ++s8) {    // 16 head dimensions per instruction: 32 bytes inside a box row
-                    const uint32_t off = (s8 >> 2) * kBoxBytes + (s8 & 3) * 32;
-                    umma_bf16(tmem_base + kColS + buf * 128, smem_desc(q_addr + off, 16, 1024),
-                              smem_desc(k_addr + off, 16, 1024), idesc_s, s8 > 0);
-                }
-                umma_commit(&bars->s_full[buf]);
-                umma_commit(&bars->k_empty[ks]);
-                ++kr.count;
-                ++sb.count;
-                return true;
-            };
-            for (int u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
-                for (int qt = 0; qt < n_qt && ok; ++qt) {
-                    const int nkb = key_tiles(qt);
-                    const uint32_t qs = qr.stage(2);
-                    ok = wait_bar(&bars->q_full[qs], qr.parity(2), abort_flag, p.status, limit);
-                    q_addr = smem_u32(smem + kOffQ + qs * kOperandBytes);
-                    // pass A: logits only
-                    for (int kb = 0; kb < nkb && ok; ++kb) ok = issue_s();
-                    if (!ok) break;
-                    // pass B: logits two tiles ahead, O += P V behind the softmax
-                    const uint32_t first_buf = sb.stage(2);         // buffer of this pass's key tile 0
-                    ok = issue_s();
-                    if (ok && nkb > 1) ok = issue_s();
-                    for (int kb = 0; kb < nkb && ok; ++kb) {
-                        const uint32_t buf = (first_buf + kb) & 1u, vs = vr.stage(kVStages);
-                        ok = wait_bar(&bars->p_full[buf], p_cnt[buf] & 1u, abort_flag, p.status, limit) &&
-                             wait_bar(&bars->v_full[vs], vr.parity(kVStages), abort_flag, p.status, limit);
-                        if (ok && kb == 0) ok = wait_bar(&bars->o_empty, (o_uses & 1u) ^ 1u, abort_flag, p.status, limit);
-                        if (!ok) break;
+            uint32_t spins = 0;
+            uint64_t t_start = 0;
+            while (o_more) {
+                bool issued = false;
+                uint64_t* nap_bar = nullptr;        // a barrier whose phase one of the cursors is waiting for
+                uint32_t nap_parity = 0;
+                {
+                    // ---- O += P V for key tile o_kb, once P is there (and V, and for the first tile the old O is out)
+                    const uint32_t buf = o_job & 1u, vs = vr.stage(kVStages);
+                    const uint32_t p_par = (buf ? p_cnt1 : p_cnt0) & 1u;
+                    if (!mbar_test_wait(&bars->p_full[buf], p_par)) {
+                        nap_bar = &bars->p_full[buf];
+                        nap_parity = p_par;
+                    } else if (!mbar_test_wait(&bars->v_full[vs], vr.parity(kVStages))) {
+                        nap_bar = &bars->v_full[vs];
+                        nap_parity = vr.parity(kVStages);
+                    } else if (o_kb == 0 && !mbar_test_wait(&bars->o_empty, (o_uses & 1u) ^ 1u)) {
+                        nap_bar = &bars->o_empty;
+                        nap_parity = (o_uses & 1u) ^ 1u;
+                    } else {
                         tmem_fence_after_sync();
                         const uint32_t v_addr = smem_u32(smem + kOffV + vs * kOperandBytes);
                         const uint32_t p_col = tmem_base + kColS + buf * 128;
@@ -420,18 +441,91 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         for (int s8 = 0; s8 < 8; ++s8) {            // 16 keys per instruction; P = hi + lo, two products
                             const uint64_t v_desc = smem_desc(v_addr + s8 * 2048, kBoxBytes, 1024);
                             const uint32_t a_col = p_col + (s8 >> 1) * 32 + (s8 & 1) * 8;
-                            umma_bf16_ts(tmem_o, a_col, v_desc, idesc_o, (kb > 0 || s8 > 0));
+                            umma_bf16_ts(tmem_o, a_col, v_desc, idesc_o, (o_kb > 0 || s8 > 0));
                             umma_bf16_ts(tmem_o, a_col + 16, v_desc, idesc_o, 1u);
                         }
                         umma_commit(&bars->v_empty[vs]);
                         ++vr.count;
-                        ++p_cnt[buf];
-                        if (kb + 2 < nkb) ok = issue_s();           // executes after the product above: same columns
+                        if (buf) ++p_cnt1; else ++p_cnt0;
+                        ++o_job;
+                        if (++o_kb == o_nkb) {
+                            umma_commit(&bars->o_full);             // the query tile's output is complete
+                            ++o_uses;
+                            o_kb = 0;
+                            if (++o_qt == n_qt) {
+                                o_qt = 0;
+                                o_u += gridDim.x;
+                                o_more = o_u < p.units;
+                            }
+                            o_nkb = key_tiles(o_qt);
+                            o_job += (uint32_t)o_nkb;               // past the next query tile's pass A jobs
+                        }
+                        issued = true;
                     }
-                    if (!ok) break;
-                    umma_commit(&bars->o_full);
-                    ++qr.count;
-                    ++o_uses;
+                }
+                if (!issued && s_more && sb.count <= o_job + 1) {
+                    // ---- S[buffer] = Q K^T for the S cursor's job.  The buffer's previous job (two back) is behind:
+                    // the softmax warps have let go of it and, where they left P there, the product that reads
+                    // it was issued above, earlier.
+                    const uint32_t ks = kr.stage(kKStages), buf = sb.stage(2), qs = sq.stage(2);
+                    const bool new_tile = s_pass == 0 && s_kb == 0;
+                    // (what the logits wait for comes sooner than P wherever both are missing)
+                    if (!mbar_test_wait(&bars->s_empty[buf], sb.parity(2) ^ 1u)) {
+                        nap_bar = &bars->s_empty[buf];
+                        nap_parity = sb.parity(2) ^ 1u;
+                    } else if (!mbar_test_wait(&bars->k_full[ks], kr.parity(kKStages))) {
+                        nap_bar = &bars->k_full[ks];
+                        nap_parity = kr.parity(kKStages);
+                    } else if (new_tile && !mbar_test_wait(&bars->q_full[qs], sq.parity(2))) {
+                        nap_bar = &bars->q_full[qs];
+                        nap_parity = sq.parity(2);
+                    } else {
+                        if (new_tile) q_addr = smem_u32(smem + kOffQ + qs * kOperandBytes);
+                        tmem_fence_after_sync();
+                        const uint32_t k_addr = smem_u32(smem + kOffK + ks * kOperandBytes);
+#pragma unroll
+                        for (int s8 = 0; s8 < 8; ++s8) {    // 16 head dimensions per instruction: 32 bytes inside a box row
+                            const uint32_t off = (s8 >> 2) * kBoxBytes + (s8 & 3) * 32;
+                            umma_bf16(tmem_base + kColS + buf * 128, smem_desc(q_addr + off, 16, 1024),
+                                      smem_desc(k_addr + off, 16, 1024), idesc_s, s8 > 0);
+                        }
+                        umma_commit(&bars->s_full[buf]);
+                        umma_commit(&bars->k_empty[ks]);
+                        ++kr.count;
+                        ++sb.count;
+                        if (++s_kb == s_nkb) {
+                            s_kb = 0;
+                            if (++s_pass == 2) {
+                                s_pass = 0;
+                                ++sq.count;
+                                if (++s_qt == n_qt) {
+                                    s_qt = 0;
+                                    s_u += gridDim.x;
+                                    s_more = s_u < p.units;
+                                }
+                                s_nkb = key_tiles(s_qt);
+                            }
+                        }
+                        issued = true;
+                    }
+                }
+                if (issued) {
+                    spins = 0;
+                    t_start = 0;
+                    continue;
+                }
+                mbar_nap(nap_bar, nap_parity, 400);
+                if ((++spins & 0x3F) == 0) {
+                    // nothing could be issued for a while: give up on another role's abort or on the time limit
+                    if (*abort_flag) break;
+                    const uint64_t now = global_timer_ns();
+                    if (t_start == 0) {
+                        t_start = now;
+                    } else if (now - t_start > limit) {
+                        *abort_flag = 1;
+                        atomicOr(p.status, kStatusWaitTimeout);
+                        break;
+                    }
                 }
             }
             // every MMA issued by this thread is complete before tensor memory goes back
@@ -458,6 +552,35 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
         auto wait_on = [&](uint64_t* bar, uint32_t parity) {
             if (!dead) dead = !wait_bar(bar, parity, abort_flag, p.status, limit);
         };
+        // ---- a query tile's attention output: bf16 into the tile's own Q slot (its MMAs are done), in the swizzled
+        // layout a TMA store expects; the producer warp sends it off before it refills the slot.
+        auto write_output = [&](uint32_t slot) {
+            wait_on(&bars->o_full, o_uses & 1u);
+            tmem_fence_after_sync();
+            {
+                float x[32];
+                tmem_ld32(tmem_row + kColO + c * 32, x);
+                tmem_wait_ld();
+                tmem_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars->o_empty);     // the accumulator is in registers
+                uint8_t* orow = smem + kOffQ + slot * kOperandBytes + (c >> 1) * kBoxBytes + row * 128;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint4 w;
+                    w.x = pack_bf16(x[8 * ch + 0], x[8 * ch + 1]);
+                    w.y = pack_bf16(x[8 * ch + 2], x[8 * ch + 3]);
+                    w.z = pack_bf16(x[8 * ch + 4], x[8 * ch + 5]);
+                    w.w = pack_bf16(x[8 * ch + 6], x[8 * ch + 7]);
+                    const int chunk = (c & 1) * 4 + ch;
+                    *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 7)) << 4)) = w;
+                }
+            }
+            fence_proxy_async();                // the store reads shared memory through the async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->out_ready[slot]);
+            ++o_uses;
+        };
         for (int u = blockIdx.x; u < p.units; u += gridDim.x) {
             const size_t srow = (size_t)u * p.capacity;
             const bool dumping = p.dump != nullptr && u >= p.dump_begin && u < p.dump_begin + p.dump_count;
@@ -477,6 +600,9 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         float x[32];
                         tmem_ld32(tmem_row + kColS + buf * 128 + c * 32, x);
                         tmem_wait_ld();
+                        tmem_fence_before_sync();   // the logits are in registers: the buffer can be refilled
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->s_empty[buf]);
                         const int key0 = kb * kTile + c * 32;
                         if (key0 + 31 > pos) {      // only the tile on the diagonal has keys beyond the row's position
 #pragma unroll
@@ -509,10 +635,10 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                             unpack2(l23, l2, l3);
                             l += (l0 + l1) + (l2 + l3);
                         }
+                    } else {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&bars->s_empty[buf]);
                     }
-                    tmem_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars->s_empty[buf]);
                 }
                 // the other parts of the row's columns: combine the four (maximum, sum) pairs
                 tmem_st4(tmem_ml + 4 * c, m, l, 0.f, 0.f);
@@ -650,34 +776,7 @@ prompt_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__
                         p.tsm[srow + own_key] = make_int2(ts, mri);
                     }
                 }
-                // ---- the tile's attention output: bf16 into the tile's own Q slot (its MMAs are done), in the
-                // swizzled layout a TMA store expects; the producer warp sends it off before it refills the slot ----
-                wait_on(&bars->o_full, o_uses & 1u);
-                tmem_fence_after_sync();
-                {
-                    float x[32];
-                    tmem_ld32(tmem_row + kColO + c * 32, x);
-                    tmem_wait_ld();
-                    tmem_fence_before_sync();
-                    uint8_t* orow = smem + kOffQ + qr.stage(2) * kOperandBytes + (c >> 1) * kBoxBytes + row * 128;
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        uint4 w;
-                        w.x = pack_bf16(x[8 * ch + 0], x[8 * ch + 1]);
-                        w.y = pack_bf16(x[8 * ch + 2], x[8 * ch + 3]);
-                        w.z = pack_bf16(x[8 * ch + 4], x[8 * ch + 5]);
-                        w.w = pack_bf16(x[8 * ch + 6], x[8 * ch + 7]);
-                        const int chunk = (c & 1) * 4 + ch;
-                        *reinterpret_cast<uint4*>(orow + ((chunk ^ (row & 7)) << 4)) = w;
-                    }
-                }
-                fence_proxy_async();                // the store reads shared memory through the async proxy
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(&bars->o_empty);
-                    mbar_arrive(&bars->out_ready[qr.stage(2)]);
-                }
-                ++o_uses;
+                write_output(qr.stage(2));
             }
         }
     }
@@ -766,6 +865,7 @@ cudaError_t prompt_launch(const Geometry& geo, StateView st, const PromptArgs& a
     p.dump_begin = a.dump_begin;
     p.dump_count = a.dump_count;
     p.wait_limit_ns = a.wait_limit_ns;
+    p.stop_after_tiles = a.stop_after_tiles;
     const int blocks = geo.units < num_sms ? geo.units : num_sms;
     return gp == 4 ? launch_gp<4>(mq, mk, mv, mo, p, blocks, stream) : launch_gp<8>(mq, mk, mv, mo, p, blocks, stream);
 }

@@ -523,6 +523,42 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_handle_recovers():
     assert du["device_status"] == 0 and used.info().evictions == fresh.info().evictions + 0
 
 
+def test_a_bounded_wait_that_runs_out_in_the_prompt_kernel_is_reported_and_the_handle_recovers():
+    """The same for the tiled prompt kernel: its producer thread stops after two key tiles (the
+    diagnostic switch), the thread that issues the tensor-core products and the softmax warps wait for
+    a tile that never comes, give up after the wait limit, and the kernel ends by itself with the
+    status word set.  After lazyev_reset the handle observes a prompt with the results of a fresh one."""
+    from tests.harness import make_engine
+    cfg = traces.tiny_config(batch=1, layers=1, prefill=300, budget=400)          # 2 units, 19 query tiles each
+    shape = (cfg.layers, cfg.batch, cfg.kv_heads, cfg.prefill, 128)
+    used, fresh = make_engine(cfg), make_engine(cfg)
+    used.set_wait_limit(0.004)
+    gen = traces.TraceGen(cfg, 42, device="cuda")
+    k, v = gen.prefill()
+    g = torch.Generator().manual_seed(6)
+    q = torch.randn(cfg.prefill, cfg.units, cfg.group, 128, generator=g).to(torch.bfloat16).cuda()
+    out_u = torch.zeros(cfg.prefill, cfg.units, cfg.group, 128, dtype=torch.bfloat16, device="cuda")
+    out_f = torch.zeros_like(out_u)
+    used.debug_starve_page_ring(2)
+    used.prefill_observed(q, k.view(shape), v.view(shape), out_u)      # queued; the kernel gives up after ~4 ms
+    with pytest.raises(binding.LazyEvError) as e:
+        used.synchronize()
+    assert e.value.code == binding.EDEVICE
+    assert used.counters().device_status & 1                  # "a bounded wait gave up"
+    torch.cuda.synchronize()                                  # the context is alive
+    used.debug_starve_page_ring(-1)
+    used.reset()
+    assert used.counters().device_status == 0
+    used.prefill_observed(q, k.view(shape), v.view(shape), out_u)
+    fresh.prefill_observed(q, k.view(shape), v.view(shape), out_f)
+    used.synchronize(); fresh.synchronize()
+    assert torch.equal(out_u, out_f)
+    du, df = used.dump_state(kv=True), fresh.dump_state(kv=True)
+    for key in ("pos", "ts", "mri", "pbar", "k", "v"):
+        assert np.array_equal(du[key], df[key]), key
+    assert du["device_status"] == 0
+
+
 @pytest.mark.parametrize("splits", [0, 1, 3])
 def test_append_inside_the_decode_launch_matches_the_separate_launch(splits):
     """Small problems write the new token inside the decode launch (one launch less per step); with the
